@@ -1,0 +1,331 @@
+"""CPU fp64 oracle for HilbertA sparse attention.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain restatement of what the method computes, written
+from the paper's definitions.  It shares no code with the CUDA library and is
+never imported by it; only the tests, the smoke check and the benchmark's CPU
+baseline call it.  Everything works on the ORIGINAL token order
+
+    [ text tokens 0..n_text ) ++ [ image tokens, row-major: n_text + r*W + c ]
+
+and in float64.
+
+Where each piece comes from
+---------------------------
+* hilbert_d2t / hilbert_t2d : the bijection pi and its inverse (Sec. 3.1, the
+  graph model of the grid and "a bijection pi that visits each cell once").
+  The paper names the Hilbert curve but fixes no orientation; the recursion
+  below (start at row 0 / col 0, end at row 0 / col W-1) is this build's
+  reading.  Parity between the eight orientations is unpinned by the paper.
+* shared_cells : the fixed central region (Sec. 3.3).
+* group_of : tile id of a Hilbert index at a given slide (Sec. 3.2, the
+  formula for q_i(l)), read as "two tokens see each other iff their q_i(l)
+  agree" -- the only reading that reproduces the ERF law of the same section.
+* mask : tiles + shared region + text rule (Sec. 3.2, Sec. 3.3, Appendix A:
+  text tokens are treated exactly like the shared anchor region).
+* attention : softmax(s * q k^T restricted to the mask) v, the quantity
+  Algorithm 1's online softmax reaches up to rounding.
+* plan arrays : the memory layout of Appendix A (prefix of text + shared
+  tokens, then the remaining image tokens in Hilbert order) and the contiguous
+  key ranges of each slid tile ("pointer shift", modular indexing, Sec. 3.2/3.4).
+
+Pins (tests/test_oracle_*.py): bijection, 4-neighbour steps, aligned-block
+squares, mirror law, an independent bit-pair construction, hand-derived 4x4 and
+8x8 tables, mask symmetry/diagonal/row counts, the ERF law, periodicity in the
+offset, reduction to dense attention (checked against torch SDPA in fp64), the
+block-diagonal case, brute-force masks on tiny grids, Table 1's GFLOPs column.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+# --------------------------------------------------------------------------
+# Sec. 3.1 -- Hilbert bijection on a 2^k x 2^k grid
+# --------------------------------------------------------------------------
+
+
+def hilbert_points(k: int):
+    """Curve of order k as a list of (x, y) = (col, row), by self-similarity.
+
+    C_0 = [(0,0)].  With s = 2^(k-1), C_k is four copies of C_(k-1):
+    transposed in the top-left quadrant, plain in the bottom-left, plain in
+    the bottom-right, anti-transposed in the top-right.
+    """
+    pts = [(0, 0)]
+    for level in range(1, k + 1):
+        s = 1 << (level - 1)
+        q0 = [(y, x) for (x, y) in pts]
+        q1 = [(x, y + s) for (x, y) in pts]
+        q2 = [(x + s, y + s) for (x, y) in pts]
+        q3 = [(2 * s - 1 - y, s - 1 - x) for (x, y) in pts]
+        pts = q0 + q1 + q2 + q3
+    return pts
+
+
+def _log2_exact(n: int) -> int:
+    k = int(n).bit_length() - 1
+    if n < 1 or (1 << k) != n:
+        raise ValueError(f"{n} is not a power of two")
+    return k
+
+
+def hilbert_d2t(H: int, W: int) -> np.ndarray:
+    """d -> row-major cell id r*W + c (pi of Sec. 3.1). int32[HW]."""
+    if H != W:
+        raise ValueError("square power-of-two grids only")
+    k = _log2_exact(H)
+    pts = hilbert_points(k)
+    return np.array([y * W + x for (x, y) in pts], dtype=np.int32)
+
+
+def hilbert_t2d(H: int, W: int) -> np.ndarray:
+    """row-major cell id -> Hilbert index d (pi^-1). int32[HW]."""
+    d2t = hilbert_d2t(H, W)
+    t2d = np.empty_like(d2t)
+    t2d[d2t] = np.arange(d2t.size, dtype=np.int32)
+    return t2d
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3 -- central shared region
+# --------------------------------------------------------------------------
+
+
+def shared_cells(H: int, W: int, shared_region: int) -> np.ndarray:
+    """Row-major ids of the centred shared_region x shared_region block."""
+    hs = int(shared_region)
+    if hs == 0:
+        return np.zeros(0, dtype=np.int32)
+    if hs < 0 or hs > H or hs > W or hs % 2:
+        raise ValueError("shared_region must be even and fit the grid")
+    r0 = H // 2 - hs // 2
+    c0 = W // 2 - hs // 2
+    cells = [r * W + c for r in range(r0, r0 + hs) for c in range(c0, c0 + hs)]
+    return np.array(cells, dtype=np.int32)
+
+
+def shared_hilbert_indices(H: int, W: int, shared_region: int) -> np.ndarray:
+    """Sorted Hilbert indices of the shared cells."""
+    t2d = hilbert_t2d(H, W)
+    return np.sort(t2d[shared_cells(H, W, shared_region)]).astype(np.int32)
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.2 -- tiles and the sliding schedule
+# --------------------------------------------------------------------------
+
+
+def group_of(d, layer_offset: int, HW: int, tile: int):
+    """q_i(l) = floor((i + l*Delta) / N_T) mod T with l*Delta = layer_offset."""
+    if tile < 1 or HW % tile:
+        raise ValueError("tile must divide H*W")
+    T = HW // tile
+    d = np.asarray(d, dtype=np.int64)
+    return ((d + int(layer_offset)) // tile) % T
+
+
+def token_classes(H, W, tile, layer_offset, shared_region, n_text):
+    """Per original token: is_global (uint8[S]) and group (int32[S], -1 = text).
+
+    Text tokens and shared-region tokens are global (Appendix A / Sec. 3.3);
+    every image token, shared or not, has a tile id from its Hilbert index.
+    """
+    HW = H * W
+    S = n_text + HW
+    t2d = hilbert_t2d(H, W)
+    is_global = np.zeros(S, dtype=np.uint8)
+    is_global[:n_text] = 1
+    is_global[n_text + shared_cells(H, W, shared_region)] = 1
+    group = np.full(S, -1, dtype=np.int32)
+    group[n_text:] = group_of(t2d, layer_offset, HW, tile).astype(np.int32)
+    return is_global, group
+
+
+def mask(H, W, tile, layer_offset, shared_region, n_text) -> np.ndarray:
+    """Boolean S x S mask over original token indices.
+
+    M[i,j] = 1 iff i is global, or j is global, or i and j are image tokens
+    of the same slid tile.
+    """
+    is_global, group = token_classes(H, W, tile, layer_offset, shared_region, n_text)
+    g = is_global.astype(bool)
+    img = group >= 0
+    same = (group[:, None] == group[None, :]) & img[:, None] & img[None, :]
+    return g[:, None] | g[None, :] | same
+
+
+def mask_row(i, is_global, group) -> np.ndarray:
+    """Row i of the mask (bool[S]) from the per-token classes."""
+    if is_global[i]:
+        return np.ones(is_global.shape[0], dtype=bool)
+    return is_global.astype(bool) | ((group == group[i]) & (group >= 0))
+
+
+def nnz(H, W, tile, layer_offset, shared_region, n_text) -> int:
+    """Number of ones in the mask, as the sum of the row counts."""
+    is_global, group = token_classes(H, W, tile, layer_offset, shared_region, n_text)
+    S = is_global.size
+    n_global = int(is_global.sum())
+    nonshared_img = (group >= 0) & (is_global == 0)
+    T = (H * W) // tile
+    per_group = np.bincount(group[nonshared_img], minlength=T).astype(np.int64)
+    total = n_global * S
+    # a non-global row sees every global column plus the non-global members of its tile
+    total += int((per_group * (n_global + per_group)).sum())
+    return total
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1's result -- masked softmax attention, fp64
+# --------------------------------------------------------------------------
+
+
+def attention(q, k, v, M, scale=None, return_lse=False):
+    """O = softmax(scale * Q K^T + log M) V per (batch, head), in float64.
+
+    q, k, v: [B, heads, S, D] in the original token order; M: bool [S, S].
+    LSE_i = max + ln(sum exp) of the scaled, masked logits (natural log).
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    B, Hh, S, D = q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty_like(q)
+    lse = np.empty((B, Hh, S), dtype=np.float64)
+    for b in range(B):
+        for h in range(Hh):
+            logits = scale * (q[b, h] @ k[b, h].T)
+            logits = np.where(M, logits, -np.inf)
+            m = logits.max(axis=1, keepdims=True)
+            p = np.exp(logits - m)
+            l = p.sum(axis=1, keepdims=True)
+            out[b, h] = (p @ v[b, h]) / l
+            lse[b, h] = (m + np.log(l))[:, 0]
+    return (out, lse) if return_lse else out
+
+
+def attention_rows(q, k, v, is_global, group, rows, scale=None):
+    """Output rows `rows` only: [B, heads, len(rows), D] fp64.
+
+    Each row is computed from its own mask row, so this scales to the largest
+    configurations when only sampled rows are wanted.
+    """
+    B, Hh, S, D = q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    out = np.empty((B, Hh, len(rows), D), dtype=np.float64)
+    for n, i in enumerate(rows):
+        cols = np.nonzero(mask_row(int(i), is_global, group))[0]
+        for b in range(B):
+            for h in range(Hh):
+                kk = np.asarray(k[b, h, cols], dtype=np.float64)
+                vv = np.asarray(v[b, h, cols], dtype=np.float64)
+                qq = np.asarray(q[b, h, int(i)], dtype=np.float64)
+                logits = scale * (kk @ qq)
+                p = np.exp(logits - logits.max())
+                out[b, h, n] = (p @ vv) / p.sum()
+    return out
+
+
+# --------------------------------------------------------------------------
+# Appendix A layout and the per-tile key ranges (canonical plan arrays)
+# --------------------------------------------------------------------------
+
+
+def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
+    """Canonical integer arrays a plan must reproduce bit for bit.
+
+    physical order = [text | shared image tokens by ascending Hilbert index |
+    non-shared image tokens by ascending Hilbert index].
+
+    windows[w] = (lo, seg0_start, seg0_len, seg1_start, seg1_len): tile w of
+    the slid partition covers Hilbert indices [lo, lo + tile) modulo HW; its
+    non-shared members occupy one or (if it wraps) two contiguous physical
+    ranges.  seg0 is the range that starts at lo.  Empty ranges are (0, 0).
+    """
+    HW = H * W
+    S = n_text + HW
+    T = HW // tile
+    if tile < 1 or HW % tile:
+        raise ValueError("tile must divide H*W")
+    d2t = hilbert_d2t(H, W)
+    t2d = hilbert_t2d(H, W)
+    sh = shared_hilbert_indices(H, W, shared_region)
+    n_sh = sh.size
+    P = n_text + n_sh
+    is_sh = np.zeros(HW, dtype=bool)
+    is_sh[sh] = True
+
+    phys2orig = np.empty(S, dtype=np.int32)
+    phys2orig[:n_text] = np.arange(n_text)
+    phys2orig[n_text:P] = n_text + d2t[sh]
+    phys2orig[P:] = n_text + d2t[~is_sh]
+    orig2phys = np.empty(S, dtype=np.int32)
+    orig2phys[phys2orig] = np.arange(S, dtype=np.int32)
+
+    # maximal runs of consecutive shared Hilbert indices
+    runs = []
+    for d in sh.tolist():
+        if runs and runs[-1][0] + runs[-1][1] == d:
+            runs[-1][1] += 1
+        else:
+            runs.append([d, 1])
+    shared_runs = np.array(runs, dtype=np.int32).reshape(-1, 2)
+
+    # c[d] = number of non-shared Hilbert indices below d, d in [0, HW]
+    c = np.concatenate([[0], np.cumsum(~is_sh)]).astype(np.int64)
+    o = int(layer_offset) % HW
+    windows = np.zeros((T, 5), dtype=np.int32)
+    for w in range(T):
+        lo = (w * tile - o) % HW
+        hi = lo + tile
+        if hi <= HW:
+            segs = [(lo, hi)]
+        else:
+            segs = [(lo, HW), (0, hi - HW)]
+        row = [lo]
+        for (a, b) in segs:
+            n = int(c[b] - c[a])
+            row += [int(P + c[a]), n] if n > 0 else [0, 0]
+        row += [0, 0] * (2 - len(segs))
+        windows[w] = row
+    return {
+        "hil_d2t": d2t,
+        "hil_t2d": t2d,
+        "phys2orig": phys2orig,
+        "orig2phys": orig2phys,
+        "shared_runs": shared_runs,
+        "windows": windows,
+        "nnz": nnz(H, W, tile, layer_offset, shared_region, n_text),
+        "n_shared": int(n_sh),
+        "prefix": int(P),
+    }
+
+
+def permute_rows(x, phys2orig):
+    """dst[b, p, :] = src[b, phys2orig[p], :] (entry gather, Sec. 3.4)."""
+    return np.ascontiguousarray(np.asarray(x)[:, phys2orig])
+
+
+def unpermute_rows(x, phys2orig):
+    """dst[b, phys2orig[p], :] = src[b, p, :] (exit gather, Sec. 3.4)."""
+    x = np.asarray(x)
+    out = np.empty_like(x)
+    out[:, phys2orig] = x
+    return out
+
+
+# --------------------------------------------------------------------------
+# error metrics used by the parity tests
+# --------------------------------------------------------------------------
+
+
+def max_abs_err(got, ref) -> float:
+    return float(np.max(np.abs(np.asarray(got, dtype=np.float64) - np.asarray(ref, dtype=np.float64))))
+
+
+def rel_l2_err(got, ref) -> float:
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    return float(np.linalg.norm((got - ref).ravel()) / np.linalg.norm(ref.ravel()))
