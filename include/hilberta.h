@@ -1,0 +1,183 @@
+/* hilberta.h -- C ABI of the HilbertA sparse-attention forward for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference hot path of Hilbert-curve tiled sparse
+ * attention for diffusion transformers: tokens of an H x W image grid are
+ * reordered along a Hilbert curve (Sec. 3.1), the reordered sequence is cut
+ * into tiles of N_T tokens with dense attention inside each tile, the tile
+ * boundaries slide by a per-layer offset with wrap-around (Sec. 3.2), every
+ * tile also attends to a static central shared region (Sec. 3.3), and text
+ * tokens are treated like the shared region (Appendix A).
+ *
+ * Conventions
+ *   - All functions return an int status: 0 on success, a negative
+ *     HILBERTA_ERR_* code otherwise.  Nothing throws or aborts.
+ *   - "device pointer" = memory of the CUDA device that was current when the
+ *     plan was created; "host pointer" = ordinary host memory.
+ *   - `stream` arguments are a cudaStream_t passed as void* (NULL = default
+ *     stream).
+ *   - ORIGINAL token order:  [ text 0..n_text ) ++ [ image tokens row-major,
+ *     token n_text + r*W + c ].
+ *   - PHYSICAL token order (the layout of Appendix A):
+ *       [ text | shared-region image tokens by ascending Hilbert index |
+ *         remaining image tokens by ascending Hilbert index ].
+ *     P = n_text + n_shared is the "global prefix" (the paper's N_s).
+ *   - Mask: query i may read key j iff i is in the prefix, or j is in the
+ *     prefix, or i and j are image tokens whose slid tile ids
+ *     floor(((d + layer_offset) mod HW) / tile) agree, d = Hilbert index.
+ */
+#ifndef HILBERTA_H_
+#define HILBERTA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HILBERTA_VERSION 100
+
+/* status codes */
+#define HILBERTA_OK 0
+#define HILBERTA_ERR_INVALID (-1)     /* bad argument value */
+#define HILBERTA_ERR_UNSUPPORTED (-2) /* valid in the method, not built (non-square / non power-of-two grid, head_dim) */
+#define HILBERTA_ERR_ARCH (-3)        /* current device is not compute capability 10.x */
+#define HILBERTA_ERR_CUDA (-4)        /* a CUDA call failed; see hilberta_last_cuda_error() */
+#define HILBERTA_ERR_NOMEM (-5)       /* host or device allocation failed */
+#define HILBERTA_ERR_BUFFER (-6)      /* export buffer too small; *needed is set */
+#define HILBERTA_ERR_UNBOUND (-7)     /* hilberta_forward before hilberta_plan_bind */
+#define HILBERTA_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired (see hilberta_plan_status) */
+
+/* element types */
+#define HILBERTA_BF16 0
+#define HILBERTA_FP32 1
+
+/* selectors for hilberta_plan_export */
+#define HILBERTA_EXPORT_HIL_D2T 0     /* int32[HW]   Hilbert index -> row-major cell r*W+c */
+#define HILBERTA_EXPORT_HIL_T2D 1     /* int32[HW]   row-major cell -> Hilbert index */
+#define HILBERTA_EXPORT_PHYS2ORIG 2   /* int32[S]    physical position -> original token */
+#define HILBERTA_EXPORT_ORIG2PHYS 3   /* int32[S]    original token -> physical position */
+#define HILBERTA_EXPORT_SHARED_RUNS 4 /* int32[n][2] maximal runs (start, length) of shared Hilbert indices */
+#define HILBERTA_EXPORT_WINDOWS 5     /* int32[T][5] per slid tile: lo, seg0_start, seg0_len, seg1_start, seg1_len */
+#define HILBERTA_EXPORT_NNZ 6         /* uint64[1]   number of (query, key) pairs the mask keeps */
+#define HILBERTA_EXPORT_INFO 7        /* int32[8]    H, W, tile, offset mod HW, shared_region, n_text, n_shared, T */
+
+typedef struct hilberta_plan_s hilberta_plan_t;
+
+/* Build the Hilbert permutation and the block-sparsity plan on the current device.
+ *
+ * Follows Sec. 3.1 (bijection pi between curve index and grid cell), Sec. 3.2
+ * (tile[q] = [q N_T, (q+1) N_T) and q_i(l) = floor((i + l Delta)/N_T) mod T with
+ * l Delta = layer_offset, wrap-around indexing), Sec. 3.3 (central shared
+ * region) and Appendix A (prefix layout).
+ *
+ *   H, W           image-token grid; must be equal powers of two, 1 <= H <= 1024
+ *                  (other shapes: HILBERTA_ERR_UNSUPPORTED).
+ *   tile           N_T in tokens; tile >= 1 and (H*W) % tile == 0, else ERR_INVALID.
+ *   layer_offset   slide in tokens, any integer; reduced modulo H*W (only its
+ *                  value modulo tile changes the mask).
+ *   shared_region  side of the centred square shared region in grid cells;
+ *                  0 = none; must be even and <= H, else ERR_INVALID.
+ *   n_text         number of text tokens (>= 0) placed before the image tokens.
+ *   out            receives the plan.  The library owns it; release with
+ *                  hilberta_plan_destroy.  All tables live in device memory.
+ *
+ * The LUT, the shared-region scan, the permutation and the per-tile key ranges
+ * are produced by CUDA kernels.  The call synchronises the device's default
+ * stream work it launches and may allocate.  A plan is immutable apart from
+ * hilberta_plan_bind and may be reused by any number of forward / permute calls.
+ */
+int hilberta_plan(int H, int W, int tile, int layer_offset, int shared_region, int n_text,
+                  hilberta_plan_t **out);
+
+/* Free a plan and every device table it owns.  NULL is accepted. */
+int hilberta_plan_destroy(hilberta_plan_t *plan);
+
+/* Copy one canonical table of the plan to HOST memory (for parity checks and
+ * callers that want the permutation).  `what` is a HILBERTA_EXPORT_* selector.
+ * If `needed` is non-NULL it receives the table's size in bytes.  If host_buf is
+ * NULL only the size is reported; if `bytes` is too small: ERR_BUFFER.
+ * The definitions are those of Sec. 3.1-3.3 and Appendix A as listed above. */
+int hilberta_plan_export(const hilberta_plan_t *plan, int what, void *host_buf, size_t bytes,
+                         size_t *needed);
+
+/* Fix the problem shape the plan's forward calls run on (Algorithm 1's
+ * configuration line: batch Z, heads, head dim D, softmax scale s, strides).
+ *
+ *   batch, heads   >= 1.  The same mask serves every (batch, head).
+ *   head_dim       bf16: 128.  fp32: 32, 64 or 128.  Others: ERR_UNSUPPORTED.
+ *   dtype          HILBERTA_BF16 (tensor-core kernel) or HILBERTA_FP32 (plain FMA kernel).
+ *   stride_b, stride_h, stride_s
+ *                  element strides of q, k, v and out (all four share them) for
+ *                  the batch, head and token axes; the head_dim axis is contiguous.
+ *                  0 for all three means the dense [batch, heads, S, head_dim] layout.
+ *                  bf16 needs every stride to be a multiple of 8 elements (16 bytes).
+ *   scale          softmax scale s; <= 0 selects 1/sqrt(head_dim).
+ *
+ * Builds the kernel's work list (device memory) and may allocate and synchronise.
+ * Rebinding replaces the previous binding. */
+int hilberta_plan_bind(hilberta_plan_t *plan, int batch, int heads, int head_dim, int dtype,
+                       int64_t stride_b, int64_t stride_h, int64_t stride_s, float scale);
+
+/* Sparse attention forward (Algorithm 1: one launch; for each query block the
+ * prefix keys K[0:N_s] and the keys of its own slid tile go through one online
+ * softmax; prefix queries read every key).
+ *
+ *   q, k, v   device pointers, PHYSICAL token order, layout as bound; read only.
+ *   out       device pointer, same layout, written; must not overlap q, k or v.
+ *             bf16: all four 16-byte aligned.
+ *   plan      a bound plan.
+ *   stream    the launch is asynchronous on this stream; no allocation, no
+ *             synchronisation.
+ *
+ * Errors: ERR_INVALID (NULL / misaligned pointers), ERR_UNBOUND, ERR_CUDA. */
+int hilberta_forward(const void *q, const void *k, const void *v, void *out,
+                     const hilberta_plan_t *plan, void *stream);
+
+/* Entry gather of Sec. 3.4 (reordering is one row gather through the Hilbert table):
+ *   dst[b, p, :] = src[b, phys2orig[p], :]   for b < batch, p < S.
+ * src is in ORIGINAL order, dst in PHYSICAL order; both device pointers to
+ * [batch, S, row_elems] contiguous arrays of `dtype`; rows must be a multiple of
+ * 16 bytes and both pointers 16-byte aligned; src and dst must not overlap.
+ * Asynchronous on `stream`. */
+int hilberta_permute(const void *src, void *dst, const hilberta_plan_t *plan, int batch,
+                     int row_elems, int dtype, void *stream);
+
+/* Exit gather of Sec. 3.4 (restores the original layout):
+ *   dst[b, t, :] = src[b, orig2phys[t], :]   for b < batch, t < S.
+ * Same argument rules as hilberta_permute with the roles of the orders swapped. */
+int hilberta_unpermute(const void *src, void *dst, const hilberta_plan_t *plan, int batch,
+                       int row_elems, int dtype, void *stream);
+
+/* Host-buffer form of the whole path, for callers that hold activations in host
+ * memory: copies q, k, v (HOST pointers, ORIGINAL order, dense
+ * [batch, heads, S, head_dim]) to the device, permutes them, runs the forward,
+ * unpermutes and copies the result to `out` (HOST pointer, ORIGINAL order).
+ * Uses a device workspace that the first call on a plan allocates (and
+ * hilberta_plan_destroy frees).  Requires a dense binding (strides 0).  The
+ * copies are asynchronous if the host buffers are pinned; the call returns
+ * after synchronising `stream`. */
+int hilberta_forward_host(const void *q, const void *k, const void *v, void *out,
+                          hilberta_plan_t *plan, void *stream);
+
+/* After a forward on `stream` has completed: 0, or ERR_TIMEOUT if a bounded wait
+ * inside the kernel gave up (the output is then undefined).  Synchronises the
+ * device.  Clears the flag. */
+int hilberta_plan_status(hilberta_plan_t *plan);
+
+/* Number of kernels the library has launched in this process (all entry points). */
+uint64_t hilberta_launch_count(void);
+
+/* Text for a status code (static storage). */
+const char *hilberta_status_string(int status);
+
+/* HILBERTA_VERSION of the loaded library. */
+int hilberta_version(void);
+
+/* The cudaError_t of the calling thread's last ERR_CUDA (0 if none). */
+int hilberta_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HILBERTA_H_ */

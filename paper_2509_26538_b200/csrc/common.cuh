@@ -1,0 +1,88 @@
+// Internal definitions shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "hilberta.h"
+
+namespace hilberta {
+
+extern thread_local int g_last_cuda_error;
+extern std::atomic<uint64_t> g_launches;
+
+#define HB_CUDA(expr)                                  \
+    do {                                               \
+        cudaError_t e__ = (expr);                      \
+        if (e__ != cudaSuccess) {                      \
+            ::hilberta::g_last_cuda_error = (int)e__;  \
+            return HILBERTA_ERR_CUDA;                  \
+        }                                              \
+    } while (0)
+
+#define HB_LAUNCHED()                                  \
+    do {                                               \
+        ::hilberta::g_launches.fetch_add(1);           \
+        HB_CUDA(cudaGetLastError());                   \
+    } while (0)
+
+// One slid tile of the partition (Sec. 3.2) in physical coordinates: the
+// non-shared members of Hilbert interval [lo, lo + tile) mod HW occupy seg0
+// (the part starting at lo) and, if the interval wraps, seg1.
+struct Window {
+    int lo;
+    int seg0_start, seg0_len;
+    int seg1_start, seg1_len;
+};
+
+// One unit of work of the tensor-core kernel: up to `rows` consecutive physical
+// query rows that share one key list of up to three contiguous ranges
+// (prefix, seg0, seg1; or the whole sequence for prefix rows).
+struct WorkItem {
+    int q_start;
+    int q_rows;
+    int n_seg;
+    int seg_start[3];
+    int seg_len[3];
+    int kv_blocks;  // sum over ranges of ceil(len / 128)
+};
+
+}  // namespace hilberta
+
+struct hilberta_plan_s {
+    int device;
+    int H, W, HW, k_log2;
+    int tile, offset, shared_region, n_text, n_shared, T, S, P;
+    uint64_t nnz;
+    // device tables
+    int *d_hil_d2t, *d_hil_t2d;      // [HW]
+    int *d_c;                        // [HW + 1] non-shared Hilbert indices below d
+    int *d_phys2orig, *d_orig2phys;  // [S]
+    int *d_row_window;               // [S] window id of a physical row, -1 for prefix rows
+    hilberta::Window *d_windows;     // [T]
+    // host mirrors of the small tables
+    std::vector<hilberta::Window> h_windows;
+    std::vector<int> h_shared_runs;  // (start, len) pairs
+    // binding
+    bool bound;
+    int batch, heads, head_dim, dtype;
+    int64_t stride_b, stride_h, stride_s;
+    float scale;
+    hilberta::WorkItem *d_work;
+    int n_work;
+    int *d_status;  // [4] error word + diagnostics written by bounded waits
+    // workspace of hilberta_forward_host
+    void *ws;
+    size_t ws_bytes;
+    int sm_count;
+};
+
+namespace hilberta {
+int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
+                     cudaStream_t stream);
+int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
+                     cudaStream_t stream);
+int attn_bf16_prepare(hilberta_plan_t *p);
+}  // namespace hilberta

@@ -1,0 +1,412 @@
+// Hilbert LUT generator, physical permutation and per-tile key ranges (device
+// kernels), plus the plan object's host-side life cycle and table export.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace hilberta {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<uint64_t> g_launches{0};
+
+// ---------------------------------------------------------------------------
+// Sec. 3.1: grid cell -> Hilbert index, one thread per cell.
+// Walk the bit planes of (col, row) from the most significant one down; each
+// plane contributes a quadrant digit and re-orients the remaining sub-square.
+// The orientation (start at row 0 / col 0, end at row 0 / col W-1) is the one
+// the library documents.  Also flags the cells of the central shared square
+// (Sec. 3.3), indexed by Hilbert index.
+// ---------------------------------------------------------------------------
+__global__ void hilbert_lut_kernel(int k, int *__restrict__ d2t, int *__restrict__ t2d,
+                                   unsigned char *__restrict__ shared_by_d, int sh_lo, int sh_hi) {
+    const int n = 1 << k;
+    const int cell = blockIdx.x * blockDim.x + threadIdx.x;
+    if (cell >= n * n) return;
+    const int row = cell >> k, col = cell & (n - 1);
+    int x = col, y = row;
+    int d = 0;
+    for (int s = n >> 1; s > 0; s >>= 1) {
+        const int rx = (x & s) ? 1 : 0;
+        const int ry = (y & s) ? 1 : 0;
+        d += s * s * ((3 * rx) ^ ry);
+        if (ry == 0) {
+            if (rx == 1) {
+                x = n - 1 - x;
+                y = n - 1 - y;
+            }
+            const int t = x;
+            x = y;
+            y = t;
+        }
+    }
+    t2d[cell] = d;
+    d2t[d] = cell;
+    shared_by_d[d] = (row >= sh_lo && row < sh_hi && col >= sh_lo && col < sh_hi) ? 1 : 0;
+}
+
+// c[d] = number of non-shared Hilbert indices below d, for d in [0, HW].
+// Single block; each thread owns a contiguous slice.
+__global__ void nonshared_scan_kernel(const unsigned char *__restrict__ shared_by_d, int HW,
+                                      int *__restrict__ c) {
+    __shared__ int warp_sums[32];
+    __shared__ int carry_sh;
+    const int tid = threadIdx.x;
+    const int nthr = blockDim.x;
+    const int per = (HW + nthr - 1) / nthr;
+    const int lo = min(tid * per, HW), hi = min(lo + per, HW);
+    int local = 0;
+    for (int d = lo; d < hi; ++d) local += shared_by_d[d] ? 0 : 1;
+    // block-wide exclusive scan of `local`
+    int v = local;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int off = 1; off < 32; off <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += t;
+    }
+    if (lane == 31) warp_sums[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        int w = (lane < (nthr >> 5)) ? warp_sums[lane] : 0;
+        for (int off = 1; off < 32; off <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, w, off);
+            if (lane >= off) w += t;
+        }
+        warp_sums[lane] = w;  // inclusive over warps
+    }
+    __syncthreads();
+    int run = v - local + (warp ? warp_sums[warp - 1] : 0);
+    for (int d = lo; d < hi; ++d) {
+        c[d] = run;
+        run += shared_by_d[d] ? 0 : 1;
+    }
+    if (tid == nthr - 1) carry_sh = run;
+    __syncthreads();
+    if (tid == 0) c[HW] = carry_sh;
+}
+
+// Appendix A layout: text first, then shared tokens, then the rest, each image
+// group by ascending Hilbert index.  One thread per original token.
+__global__ void layout_kernel(int HW, int n_text, int P, int tile, int offset,
+                              const int *__restrict__ t2d, const int *__restrict__ c,
+                              const unsigned char *__restrict__ shared_by_d,
+                              int *__restrict__ phys2orig, int *__restrict__ orig2phys,
+                              int *__restrict__ row_window) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_text + HW) return;
+    if (t < n_text) {
+        phys2orig[t] = t;
+        orig2phys[t] = t;
+        row_window[t] = -1;
+        return;
+    }
+    const int d = t2d[t - n_text];
+    const int below = c[d];
+    int phys;
+    if (shared_by_d[d]) {
+        phys = n_text + (d - below);
+        row_window[phys] = -1;
+    } else {
+        phys = P + below;
+        row_window[phys] = ((d + offset) % HW) / tile;
+    }
+    phys2orig[phys] = t;
+    orig2phys[t] = phys;
+}
+
+// Sec. 3.2 with wrap-around: slid tile w covers Hilbert indices
+// [w*tile - offset, +tile) mod HW; its non-shared members are contiguous in the
+// physical order, in one range or two if the interval wraps.
+__global__ void window_kernel(int HW, int T, int tile, int offset, int P, const int *__restrict__ c,
+                              Window *__restrict__ win) {
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w >= T) return;
+    long long lo_ll = ((long long)w * tile - offset) % HW;
+    if (lo_ll < 0) lo_ll += HW;
+    const int lo = (int)lo_ll;
+    const int hi = lo + tile;
+    Window r;
+    r.lo = lo;
+    const int a0 = lo, b0 = hi <= HW ? hi : HW;
+    const int n0 = c[b0] - c[a0];
+    r.seg0_start = n0 > 0 ? P + c[a0] : 0;
+    r.seg0_len = n0;
+    r.seg1_start = 0;
+    r.seg1_len = 0;
+    if (hi > HW) {
+        const int n1 = c[hi - HW] - c[0];
+        r.seg1_start = n1 > 0 ? P + c[0] : 0;
+        r.seg1_len = n1;
+    }
+    win[w] = r;
+}
+
+static int ilog2_exact(int n) {
+    int k = 0;
+    while ((1 << k) < n) ++k;
+    return ((1 << k) == n) ? k : -1;
+}
+
+static void free_plan(hilberta_plan_t *p) {
+    if (!p) return;
+    cudaFree(p->d_hil_d2t);
+    cudaFree(p->d_hil_t2d);
+    cudaFree(p->d_c);
+    cudaFree(p->d_phys2orig);
+    cudaFree(p->d_orig2phys);
+    cudaFree(p->d_row_window);
+    cudaFree(p->d_windows);
+    cudaFree(p->d_work);
+    cudaFree(p->d_status);
+    cudaFree(p->ws);
+    delete p;
+}
+
+static int build_plan(hilberta_plan_t *p) {
+    const int HW = p->HW, S = p->S;
+    unsigned char *d_shared = nullptr;
+    HB_CUDA(cudaMalloc(&p->d_hil_d2t, sizeof(int) * HW));
+    HB_CUDA(cudaMalloc(&p->d_hil_t2d, sizeof(int) * HW));
+    HB_CUDA(cudaMalloc(&p->d_c, sizeof(int) * (HW + 1)));
+    HB_CUDA(cudaMalloc(&p->d_phys2orig, sizeof(int) * S));
+    HB_CUDA(cudaMalloc(&p->d_orig2phys, sizeof(int) * S));
+    HB_CUDA(cudaMalloc(&p->d_row_window, sizeof(int) * S));
+    HB_CUDA(cudaMalloc(&p->d_windows, sizeof(Window) * p->T));
+    HB_CUDA(cudaMalloc(&p->d_status, sizeof(int) * 4));
+    HB_CUDA(cudaMemset(p->d_status, 0, sizeof(int) * 4));
+    HB_CUDA(cudaMalloc(&d_shared, HW));
+
+    const int sh_lo = p->H / 2 - p->shared_region / 2;
+    const int sh_hi = sh_lo + p->shared_region;
+    int rc = HILBERTA_OK;
+    do {
+        hilbert_lut_kernel<<<(HW + 255) / 256, 256>>>(p->k_log2, p->d_hil_d2t, p->d_hil_t2d, d_shared,
+                                                      sh_lo, sh_hi);
+        g_launches.fetch_add(1);
+        nonshared_scan_kernel<<<1, 1024>>>(d_shared, HW, p->d_c);
+        g_launches.fetch_add(1);
+        layout_kernel<<<(S + 255) / 256, 256>>>(HW, p->n_text, p->P, p->tile, p->offset, p->d_hil_t2d,
+                                                p->d_c, d_shared, p->d_phys2orig, p->d_orig2phys,
+                                                p->d_row_window);
+        g_launches.fetch_add(1);
+        window_kernel<<<(p->T + 127) / 128, 128>>>(HW, p->T, p->tile, p->offset, p->P, p->d_c,
+                                                   p->d_windows);
+        g_launches.fetch_add(1);
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            rc = HILBERTA_ERR_CUDA;
+            break;
+        }
+        // host mirrors of the small tables
+        p->h_windows.resize(p->T);
+        std::vector<unsigned char> h_shared(HW);
+        e = cudaMemcpy(p->h_windows.data(), p->d_windows, sizeof(Window) * p->T, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) e = cudaMemcpy(h_shared.data(), d_shared, HW, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            rc = HILBERTA_ERR_CUDA;
+            break;
+        }
+        int n_sh = 0;
+        for (int d = 0; d < HW; ++d) {
+            if (!h_shared[d]) continue;
+            ++n_sh;
+            size_t n = p->h_shared_runs.size();
+            if (n && p->h_shared_runs[n - 2] + p->h_shared_runs[n - 1] == d) {
+                p->h_shared_runs[n - 1] += 1;
+            } else {
+                p->h_shared_runs.push_back(d);
+                p->h_shared_runs.push_back(1);
+            }
+        }
+        if (n_sh != p->n_shared) {
+            rc = HILBERTA_ERR_INVALID;  // cannot happen for validated arguments
+            break;
+        }
+        // kept pairs: prefix rows see everything; other rows see the prefix and
+        // the non-shared members of their own slid tile
+        const uint64_t Pq = (uint64_t)p->P, Sq = (uint64_t)S;
+        uint64_t nnz = Pq * Sq;
+        for (const Window &w : p->h_windows) {
+            const uint64_t r = (uint64_t)w.seg0_len + (uint64_t)w.seg1_len;
+            nnz += r * (Pq + r);
+        }
+        p->nnz = nnz;
+    } while (0);
+    cudaFree(d_shared);
+    return rc;
+}
+
+}  // namespace hilberta
+
+using namespace hilberta;
+
+extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int shared_region, int n_text,
+                             hilberta_plan_t **out) {
+    if (!out) return HILBERTA_ERR_INVALID;
+    *out = nullptr;
+    if (H < 1 || W < 1 || n_text < 0 || tile < 1 || shared_region < 0) return HILBERTA_ERR_INVALID;
+    if (H != W || ilog2_exact(H) < 0 || H > 1024) return HILBERTA_ERR_UNSUPPORTED;
+    const int HW = H * W;
+    if (HW % tile) return HILBERTA_ERR_INVALID;
+    if (shared_region % 2 || shared_region > H) return HILBERTA_ERR_INVALID;
+    if ((long long)n_text + HW > (1ll << 30)) return HILBERTA_ERR_INVALID;
+
+    int dev = 0;
+    HB_CUDA(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    HB_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return HILBERTA_ERR_ARCH;
+
+    hilberta_plan_t *p = new (std::nothrow) hilberta_plan_t();
+    if (!p) return HILBERTA_ERR_NOMEM;
+    p->device = dev;
+    p->sm_count = prop.multiProcessorCount;
+    p->H = H;
+    p->W = W;
+    p->HW = HW;
+    p->k_log2 = ilog2_exact(H);
+    p->tile = tile;
+    long long o = (long long)layer_offset % HW;
+    if (o < 0) o += HW;
+    p->offset = (int)o;
+    p->shared_region = shared_region;
+    p->n_text = n_text;
+    p->n_shared = shared_region * shared_region;
+    p->T = HW / tile;
+    p->S = n_text + HW;
+    p->P = n_text + p->n_shared;
+    p->bound = false;
+    int rc = build_plan(p);
+    if (rc != HILBERTA_OK) {
+        free_plan(p);
+        return rc;
+    }
+    *out = p;
+    return HILBERTA_OK;
+}
+
+extern "C" int hilberta_plan_destroy(hilberta_plan_t *plan) {
+    free_plan(plan);
+    return HILBERTA_OK;
+}
+
+extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *host_buf, size_t bytes,
+                                    size_t *needed) {
+    if (!p) return HILBERTA_ERR_INVALID;
+    size_t need = 0;
+    const void *dsrc = nullptr;
+    std::vector<int> tmp;
+    uint64_t nnz = p->nnz;
+    const void *hsrc = nullptr;
+    switch (what) {
+        case HILBERTA_EXPORT_HIL_D2T: need = sizeof(int) * p->HW; dsrc = p->d_hil_d2t; break;
+        case HILBERTA_EXPORT_HIL_T2D: need = sizeof(int) * p->HW; dsrc = p->d_hil_t2d; break;
+        case HILBERTA_EXPORT_PHYS2ORIG: need = sizeof(int) * p->S; dsrc = p->d_phys2orig; break;
+        case HILBERTA_EXPORT_ORIG2PHYS: need = sizeof(int) * p->S; dsrc = p->d_orig2phys; break;
+        case HILBERTA_EXPORT_SHARED_RUNS:
+            need = sizeof(int) * p->h_shared_runs.size();
+            hsrc = p->h_shared_runs.data();
+            break;
+        case HILBERTA_EXPORT_WINDOWS:
+            need = sizeof(Window) * p->h_windows.size();
+            hsrc = p->h_windows.data();
+            break;
+        case HILBERTA_EXPORT_NNZ: need = sizeof(uint64_t); hsrc = &nnz; break;
+        case HILBERTA_EXPORT_INFO:
+            tmp = {p->H, p->W, p->tile, p->offset, p->shared_region, p->n_text, p->n_shared, p->T};
+            need = sizeof(int) * tmp.size();
+            hsrc = tmp.data();
+            break;
+        default: return HILBERTA_ERR_INVALID;
+    }
+    if (needed) *needed = need;
+    if (!host_buf) return HILBERTA_OK;
+    if (bytes < need) return HILBERTA_ERR_BUFFER;
+    if (dsrc) {
+        HB_CUDA(cudaMemcpy(host_buf, dsrc, need, cudaMemcpyDeviceToHost));
+    } else if (need) {
+        memcpy(host_buf, hsrc, need);
+    }
+    return HILBERTA_OK;
+}
+
+extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int head_dim, int dtype,
+                                  int64_t stride_b, int64_t stride_h, int64_t stride_s, float scale) {
+    if (!p || batch < 1 || heads < 1 || head_dim < 1) return HILBERTA_ERR_INVALID;
+    if (dtype != HILBERTA_BF16 && dtype != HILBERTA_FP32) return HILBERTA_ERR_INVALID;
+    if (dtype == HILBERTA_BF16 && head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
+    if (dtype == HILBERTA_FP32 && head_dim != 32 && head_dim != 64 && head_dim != 128)
+        return HILBERTA_ERR_UNSUPPORTED;
+    if (stride_b == 0 && stride_h == 0 && stride_s == 0) {
+        stride_s = head_dim;
+        stride_h = (int64_t)p->S * head_dim;
+        stride_b = (int64_t)heads * stride_h;
+    }
+    if (stride_b <= 0 || stride_h <= 0 || stride_s < head_dim) return HILBERTA_ERR_INVALID;
+    if (dtype == HILBERTA_BF16 && ((stride_b | stride_h | stride_s) & 7)) return HILBERTA_ERR_INVALID;
+    if ((int64_t)batch * heads > 65535) return HILBERTA_ERR_INVALID;
+    p->bound = false;
+    p->batch = batch;
+    p->heads = heads;
+    p->head_dim = head_dim;
+    p->dtype = dtype;
+    p->stride_b = stride_b;
+    p->stride_h = stride_h;
+    p->stride_s = stride_s;
+    p->scale = scale > 0.f ? scale : 1.0f / sqrtf((float)head_dim);
+    if (dtype == HILBERTA_BF16) {
+        int rc = attn_bf16_prepare(p);
+        if (rc != HILBERTA_OK) return rc;
+    }
+    p->bound = true;
+    return HILBERTA_OK;
+}
+
+extern "C" int hilberta_forward(const void *q, const void *k, const void *v, void *out,
+                                const hilberta_plan_t *p, void *stream) {
+    if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
+    if (!p->bound) return HILBERTA_ERR_UNBOUND;
+    if (out == q || out == k || out == v) return HILBERTA_ERR_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->dtype == HILBERTA_FP32) return launch_attn_fp32(p, q, k, v, out, st);
+    const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
+    if (bits & 15) return HILBERTA_ERR_INVALID;
+    return launch_attn_bf16(p, q, k, v, out, st);
+}
+
+extern "C" int hilberta_plan_status(hilberta_plan_t *p) {
+    if (!p) return HILBERTA_ERR_INVALID;
+    int h[4] = {0, 0, 0, 0};
+    HB_CUDA(cudaDeviceSynchronize());
+    HB_CUDA(cudaMemcpy(h, p->d_status, sizeof(h), cudaMemcpyDeviceToHost));
+    if (h[0] != 0) {
+        HB_CUDA(cudaMemset(p->d_status, 0, sizeof(h)));
+        return HILBERTA_ERR_TIMEOUT;
+    }
+    return HILBERTA_OK;
+}
+
+extern "C" uint64_t hilberta_launch_count(void) { return g_launches.load(); }
+
+extern "C" const char *hilberta_status_string(int status) {
+    switch (status) {
+        case HILBERTA_OK: return "ok";
+        case HILBERTA_ERR_INVALID: return "invalid argument";
+        case HILBERTA_ERR_UNSUPPORTED: return "unsupported shape";
+        case HILBERTA_ERR_ARCH: return "device is not sm_100";
+        case HILBERTA_ERR_CUDA: return "CUDA error";
+        case HILBERTA_ERR_NOMEM: return "out of memory";
+        case HILBERTA_ERR_BUFFER: return "buffer too small";
+        case HILBERTA_ERR_UNBOUND: return "plan not bound to a problem shape";
+        case HILBERTA_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int hilberta_version(void) { return HILBERTA_VERSION; }
+
+extern "C" int hilberta_last_cuda_error(void) { return g_last_cuda_error; }
