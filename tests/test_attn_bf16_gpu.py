@@ -1,0 +1,165 @@
+"""bf16 tensor-core forward parity with the fp64 oracle.
+
+Tolerance for bf16 inputs: max-abs error <= 1e-2 and relative L2 error <= 5e-3
+over the output tensor.  Small and Flux-1024 cases are compared element by
+element; the larger workloads on seeded samples of query rows (every head)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attn_c
+from oracle import hilberta_oracle as orc
+from paper_2509_26538_b200 import binding as hb
+from paper_2509_26538_b200.inputs import WORKLOADS, make_qkv, make_smooth_qkv, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+TOL_MAX_ABS = 1e-2
+TOL_REL_L2 = 5e-3
+
+
+def run_gpu(plan, q, k, v, scale=0.0, twice=True):
+    """Original-order host tensors in, original-order host tensor out; permute,
+    forward and unpermute all through the C ABI."""
+    qd, kd, vd = (t.cuda() for t in (q, k, v))
+    qp, kp, vp, od = (torch.empty_like(qd) for _ in range(4))
+    op = torch.full_like(qd, float("nan"))
+    plan.permute(qd, qp)
+    plan.permute(kd, kp)
+    plan.permute(vd, vp)
+    plan.bind_like(qp, scale)
+    plan.forward(qp, kp, vp, op)
+    assert plan.status() == 0
+    if twice:  # same launch again: results must be bit-identical
+        op2 = torch.full_like(qd, float("nan"))
+        plan.forward(qp, kp, vp, op2)
+        assert plan.status() == 0
+        assert torch.equal(op.view(torch.int16), op2.view(torch.int16))
+    plan.unpermute(op, od)
+    torch.cuda.synchronize()
+    return od.cpu()
+
+
+def check(got, ref):
+    got = got.double().numpy()
+    assert np.isfinite(got).all()
+    ma, rl = orc.max_abs_err(got, ref), orc.rel_l2_err(got, ref)
+    assert ma <= TOL_MAX_ABS and rl <= TOL_REL_L2, (ma, rl)
+    return ma, rl
+
+
+def oracle_rows(H, tile, o, hs, nt, q, k, v, rows=None, scale=None):
+    ig, grp = orc.token_classes(H, H, tile, o, hs, nt)
+    return attn_c.attention_rows(q.float().numpy(), k.float().numpy(), v.float().numpy(), ig, grp,
+                                 rows=rows, scale=scale)
+
+
+@pytest.mark.parametrize("H,tile,o,hs,nt,B,heads", [
+    (16, 64, 16, 2, 0, 1, 2),      # tiny grid, ragged 62/63/64-key ranges, wrapped tile
+    (16, 64, 0, 2, 5, 2, 2),       # text tokens, batch 2
+    (16, 256, 3, 0, 0, 1, 1),      # one tile, no prefix: dense
+    (16, 64, 0, 0, 0, 1, 2),       # block diagonal, no prefix at all
+    (8, 16, 4, 8, 0, 1, 1),        # every token shared: dense through the prefix path
+    (32, 128, 100, 4, 77, 1, 3),   # ragged prefix (93 rows), several blocks per range
+    (32, 512, 256, 8, 200, 1, 2),
+    (1, 1, 0, 0, 0, 1, 1),         # a single token
+    (2, 2, 1, 0, 300, 1, 2),       # almost only text
+])
+def test_small_cases_elementwise(H, tile, o, hs, nt, B, heads):
+    S = nt + H * H
+    g = torch.Generator().manual_seed(1000 + H * 7 + nt)
+    q, k, v = (torch.randn((B, heads, S, 128), generator=g).bfloat16() for _ in range(3))
+    plan = hb.Plan(H, H, tile, o, hs, nt)
+    try:
+        got = run_gpu(plan, q, k, v)
+    finally:
+        plan.destroy()
+    check(got, oracle_rows(H, tile, o, hs, nt, q, k, v))
+
+
+def test_dense_reduction_vs_sdpa():
+    H, nt = 16, 40
+    S = nt + H * H
+    g = torch.Generator().manual_seed(77)
+    q, k, v = (torch.randn((1, 2, S, 128), generator=g).bfloat16() for _ in range(3))
+    plan = hb.Plan(H, H, H * H, 9, 0, nt)
+    try:
+        got = run_gpu(plan, q, k, v)
+    finally:
+        plan.destroy()
+    ref = torch.nn.functional.scaled_dot_product_attention(q.double(), k.double(), v.double())
+    check(got, ref.numpy())
+
+
+def test_custom_scale_peaky_and_smooth_inputs():
+    wl = WORKLOADS["flux1024"].with_(H=32, W=32, n_text=64, heads=2, tile=256, shared_region=4, layer_offset=128)
+    for maker in (lambda: make_qkv(wl, q_gain=8.0), lambda: make_smooth_qkv(wl)):
+        q, k, v = maker()
+        plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
+        try:
+            got = run_gpu(plan, q, k, v, scale=0.05)
+        finally:
+            plan.destroy()
+        check(got, oracle_rows(wl.H, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text, q, k, v, scale=0.05))
+
+
+def test_strided_layout():
+    H, tile, o, hs, nt = 16, 64, 16, 2, 9
+    S = nt + H * H
+    g = torch.Generator().manual_seed(5)
+    q, k, v = (torch.randn((2, 3, S, 128), generator=g).bfloat16() for _ in range(3))
+    ref = oracle_rows(H, tile, o, hs, nt, q, k, v)
+    plan = hb.Plan(H, H, tile, o, hs, nt)
+    try:
+        p2o = torch.from_numpy(plan.export(hb.EXPORT_PHYS2ORIG).astype(np.int64))
+
+        def strided(t):  # [B, S, heads, D] storage viewed as [B, heads, S, D]
+            return t[:, :, p2o].permute(0, 2, 1, 3).contiguous().cuda().permute(0, 2, 1, 3)
+        qp, kp, vp = strided(q), strided(k), strided(v)
+        out = torch.empty_like(qp)
+        plan.bind_like(qp)
+        plan.forward(qp, kp, vp, out)
+        assert plan.status() == 0
+        got = torch.empty_like(q)
+        got[:, :, p2o] = out.cpu()
+    finally:
+        plan.destroy()
+    check(got, ref)
+
+
+@pytest.mark.parametrize("tile,heads", [(256, 4), (512, 4), (1024, 24)])
+def test_flux1024_elementwise(tile, heads):
+    wl = WORKLOADS["flux1024"]
+    q, k, v = make_qkv(wl, heads=heads)
+    o = tile // 2
+    plan = hb.Plan(wl.H, wl.W, tile, o, wl.shared_region, wl.n_text)
+    try:
+        got = run_gpu(plan, q, k, v)
+    finally:
+        plan.destroy()
+    check(got, oracle_rows(wl.H, tile, o, wl.shared_region, wl.n_text, q, k, v))
+
+
+@pytest.mark.parametrize("name,n_rows", [("flux2048", 160), ("flux4096", 96)])
+def test_full_size_sampled_rows(name, n_rows):
+    """Bench launch configuration (all heads, full sequence); the oracle computes
+    the sampled query rows one by one."""
+    wl = WORKLOADS[name]
+    q, k, v = make_qkv(wl)
+    plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
+    try:
+        got = run_gpu(plan, q, k, v, twice=(name == "flux2048"))
+        # rows around every tile boundary of the first two tiles as well
+        win = plan.export(hb.EXPORT_WINDOWS)
+        p2o = plan.export(hb.EXPORT_PHYS2ORIG)
+    finally:
+        plan.destroy()
+    edge = []
+    for w in win[:3]:
+        for (s, n) in ((w[1], w[2]), (w[3], w[4])):
+            if n:
+                edge += [int(p2o[s]), int(p2o[s + n - 1]), int(p2o[s + min(n - 1, 127)]), int(p2o[s + min(n - 1, 128)])]
+    rows = sorted(set(sample_rows(wl, n_rows) + edge))
+    ref = oracle_rows(wl.H, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text, q, k, v, rows=rows)
+    check(got[:, :, rows], ref)
+    assert torch.isfinite(got.float()).all()
