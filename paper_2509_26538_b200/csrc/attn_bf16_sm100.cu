@@ -3,18 +3,25 @@
 // accumulators in tensor memory, fp32 online softmax, one launch for prefix
 // rows and tile rows alike.
 //
-// A work item is up to 128 consecutive physical query rows that share a key
-// list of up to three contiguous ranges (prefix, tile range, wrapped tile
-// range -- or the whole sequence for prefix rows).  The key list is cut into
-// blocks of 128 keys; the ragged last block of a range is masked by column.
+// A work item is up to 256 consecutive physical query rows (two 128-row query
+// tiles) that share a key list of up to three contiguous ranges (prefix, tile
+// range, wrapped tile range -- or the whole sequence for prefix rows).  The
+// key list is cut into blocks of 128 keys; the ragged last block of a range is
+// masked by column.  Prefix blocks and tile blocks run through one loop with
+// one online-softmax state per row.
 //
-// Roles inside a CTA (persistent over work items):
-//   warps 0-3  softmax / correction / epilogue, thread r owns query row r
-//              (TMEM lane r)
-//   warp  4    TMA producer (one elected lane)
-//   warp  5    MMA issuer   (one elected lane)
-// TMEM columns: [0,128) S = Q K^T (fp32), overwritten in place by P (bf16,
-// columns [0,64)); [128,256) O accumulator (fp32).
+// Roles inside a CTA (one CTA per SM, persistent over work items):
+//   warps 0-3  softmax + epilogue for query tile 0, thread r owns row r (TMEM lane r)
+//   warps 4-7  softmax + epilogue for query tile 1
+//   warp  8    TMA producer (one elected lane)
+//   warp  9    MMA issuer   (one elected lane)
+//   warps 10-11 idle; their registers go to the softmax warps (setmaxnreg)
+// The two query tiles ping-pong: while one tile's softmax runs on the CUDA
+// cores, the tensor cores work on the other tile's P V and next Q K^T.
+// TMEM columns: S_t = Q_t K^T (fp32) at [128 t, 128 t + 128), overwritten in
+// place by P_t (bf16, first 64 columns); O_t accumulators at [256 + 128 t, +128).
+// The running maximum is only advanced when it grows by more than 2^8, so the
+// O accumulator is rescaled rarely; exponentials stay below 2^8.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -29,22 +36,25 @@ using namespace ptx;
 
 namespace {
 
-constexpr int BM = 128;      // query rows per work item
-constexpr int BN = 128;      // keys per block
-constexpr int HD = 128;      // head dim
-constexpr int STAGES = 2;    // K and V ring depth
-constexpr int TILE_BYTES = BN * HD * 2;   // 32 KB: two 64-column slabs of 128 rows
+constexpr int BM = 128;        // rows per query tile
+constexpr int BN = 128;        // keys per block
+constexpr int HD = 128;        // head dim
+constexpr int QT = 2;          // query tiles per work item
+constexpr int ITEM_ROWS = QT * BM;
+constexpr int NSTAGE = 5;      // K/V ring slots (K0 V0 K1 V1 ...)
+constexpr int TILE_BYTES = BN * HD * 2;  // 32 KB: two 64-column slabs of 128 rows
 constexpr int SLAB_BYTES = TILE_BYTES / 2;
-constexpr int THREADS = 192;
-constexpr int SMEM_BYTES = (1 + 2 * STAGES) * TILE_BYTES + 1024;
-constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t TM_S = 0, TM_O = 128;
+constexpr int THREADS = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle (register donors)
+constexpr int SMEM_BYTES = (QT + NSTAGE) * TILE_BYTES + 1024;
+constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_CYCLES = 2000000000ll;  // ~1 s: far beyond any legitimate wait
+constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 
 enum Bar {
-    Q_FULL = 0, Q_EMPTY, S_FULL, P_READY, O_DONE, DRAIN,
-    K_FULL, K_EMPTY = K_FULL + STAGES, V_FULL = K_EMPTY + STAGES, V_EMPTY = V_FULL + STAGES,
-    NUM_BARS = V_EMPTY + STAGES
+    Q_FULL = 0, Q_EMPTY, DRAIN,
+    S_FULL, P_READY = S_FULL + QT, PV_DONE = P_READY + QT,
+    KV_FULL = PV_DONE + QT, KV_EMPTY = KV_FULL + NSTAGE,
+    NUM_BARS = KV_EMPTY + NSTAGE
 };
 
 struct Params {
@@ -61,6 +71,7 @@ struct Params {
 // Wait with a deadline; on expiry record where and raise the CTA's abort flag.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                               int *status, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -82,6 +93,38 @@ __device__ __forceinline__ int item_blocks(const WorkItem &it, int seg) {
     return (it.seg_len[seg] + BN - 1) / BN;
 }
 
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+// S_t = Q_t K^T for one 128-key block: 8 MMAs of K = 16.
+__device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t sQt, uint32_t sKslot) {
+    constexpr uint32_t IDESC = idesc_bf16_f32(BM, BN, 0, 0);
+#pragma unroll
+    for (int k = 0; k < HD / 16; ++k) {
+        const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
+        mma_ss(tmem_s, smem_desc_sw128(sQt + off, 16, 1024), smem_desc_sw128(sKslot + off, 16, 1024), IDESC,
+               k > 0);
+    }
+}
+
+// O_t (+)= P_t V for one 128-key block: P from TMEM, V row-major in smem (N-major operand).
+__device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, bool accumulate) {
+    constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
+#pragma unroll
+    for (int k = 0; k < BN / 16; ++k) {
+        mma_ts(tmem_o, tmem_p + k * 8, smem_desc_sw128(sVslot + k * 2048, SLAB_BYTES, 1024), IDESC,
+               (accumulate || k > 0) ? 1u : 0u);
+    }
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const Params prm) {
@@ -92,18 +135,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sQ = smem_u32(smem);
-    const uint32_t sK = sQ + TILE_BYTES;
-    const uint32_t sV = sK + STAGES * TILE_BYTES;
+    const uint32_t sKV = sQ + QT * TILE_BYTES;
     const int tid = threadIdx.x, warp = tid >> 5;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int i = 0; i < NUM_BARS; ++i) mbar_init(bar(i), i == P_READY ? 128 : 1);
+        for (int i = 0; i < NUM_BARS; ++i)
+            mbar_init(bar(i), (i >= P_READY && i < P_READY + QT) ? 128 : 1);
         mbar_fence_init();
     }
-    if (warp == 4) {
+    if (warp == 8) {
         tmem_alloc(smem_u32(&tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
@@ -113,39 +156,46 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const uint32_t tmem = tmem_slot;
     const long long total = (long long)prm.n_work * prm.bh;
 
-    if (warp == 4) {
+    // registers move from the data-movement warpgroup to the two softmax warpgroups
+    if (warp >= 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    }
+    if (warp == 8) {
         // ------------------------------------------------------------ producer
         if (elect_one()) {
             prefetch_tmap(&tmQ);
             prefetch_tmap(&tmK);
             prefetch_tmap(&tmV);
-            uint32_t it = 0, qcount = 0;
+            uint32_t kvc = 0, qc = 0;
             bool ok = true;
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem wi = prm.work[w / prm.bh];
                 const int bh = (int)(w % prm.bh);
                 const int b = bh / prm.heads, h = bh % prm.heads;
-                ok = wait_or_abort(bar(Q_EMPTY), (qcount & 1) ^ 1, &abort_flag, prm.status, 0x101);
+                const int nt = wi.q_rows > BM ? 2 : 1;
+                ok = wait_or_abort(bar(Q_EMPTY), (qc & 1) ^ 1, &abort_flag, prm.status, 0x101);
                 if (!ok) break;
-                mbar_expect_tx(bar(Q_FULL), TILE_BYTES);
-                tma_load_4d(sQ, &tmQ, bar(Q_FULL), 0, wi.q_start, h, b);
-                tma_load_4d(sQ + SLAB_BYTES, &tmQ, bar(Q_FULL), 64, wi.q_start, h, b);
-                ++qcount;
+                ++qc;
+                mbar_expect_tx(bar(Q_FULL), nt * TILE_BYTES);
+                for (int t = 0; t < nt; ++t) {
+                    tma_load_4d(sQ + t * TILE_BYTES, &tmQ, bar(Q_FULL), 0, wi.q_start + t * BM, h, b);
+                    tma_load_4d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, bar(Q_FULL), 64, wi.q_start + t * BM, h, b);
+                }
                 for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                     const int nb = item_blocks(wi, seg);
-                    for (int j = 0; j < nb; ++j, ++it) {
-                        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                    for (int j = 0; j < nb; ++j) {
                         const int row = wi.seg_start[seg] + j * BN;
-                        ok = wait_or_abort(bar(K_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x102);
+#pragma unroll
+                        for (int kv = 0; kv < 2; ++kv, ++kvc) {
+                            const uint32_t s = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
+                            ok = wait_or_abort(bar(KV_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x102);
+                            if (!ok) break;
+                            const CUtensorMap *tm = kv ? &tmV : &tmK;
+                            mbar_expect_tx(bar(KV_FULL + s), TILE_BYTES);
+                            tma_load_4d(sKV + s * TILE_BYTES, tm, bar(KV_FULL + s), 0, row, h, b);
+                            tma_load_4d(sKV + s * TILE_BYTES + SLAB_BYTES, tm, bar(KV_FULL + s), 64, row, h, b);
+                        }
                         if (!ok) break;
-                        mbar_expect_tx(bar(K_FULL + s), TILE_BYTES);
-                        tma_load_4d(sK + s * TILE_BYTES, &tmK, bar(K_FULL + s), 0, row, h, b);
-                        tma_load_4d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, bar(K_FULL + s), 64, row, h, b);
-                        ok = wait_or_abort(bar(V_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x103);
-                        if (!ok) break;
-                        mbar_expect_tx(bar(V_FULL + s), TILE_BYTES);
-                        tma_load_4d(sV + s * TILE_BYTES, &tmV, bar(V_FULL + s), 0, row, h, b);
-                        tma_load_4d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, bar(V_FULL + s), 64, row, h, b);
                     }
                 }
             }
@@ -156,154 +206,173 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ---------------------------------------------------------- MMA issuer
         if (elect_one()) {
-            constexpr uint32_t IDESC_QK = idesc_bf16_f32(BM, BN, 0, 0);
-            constexpr uint32_t IDESC_PV = idesc_bf16_f32(BM, HD, 0, 1);
-            uint32_t it = 0, qcount = 0;
+            uint32_t g = 0;   // blocks consumed so far: K of block g is ring entry 2g, V is 2g + 1
+            uint32_t qc = 0;
+            uint32_t cP[QT] = {0, 0};
             bool ok = true;
+            auto slot_of = [](uint32_t e) { return e % NSTAGE; };
+            auto phase_of = [](uint32_t e) { return (e / NSTAGE) & 1; };
             for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
                 const WorkItem wi = prm.work[w / prm.bh];
-                ok = wait_or_abort(bar(Q_FULL), qcount & 1, &abort_flag, prm.status, 0x201);
+                const int nt = wi.q_rows > BM ? 2 : 1;
+                const int n = wi.kv_blocks;
+                ok = wait_or_abort(bar(Q_FULL), qc & 1, &abort_flag, prm.status, 0x201);
                 if (!ok) break;
-                ++qcount;
-                int blk = 0;
-                for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
-                    const int nb = item_blocks(wi, seg);
-                    for (int j = 0; j < nb; ++j, ++it, ++blk) {
-                        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                        ok = wait_or_abort(bar(K_FULL + s), ph, &abort_flag, prm.status, 0x202);
+                ++qc;
+                // S_t(0)
+                ok = wait_or_abort(bar(KV_FULL + slot_of(2 * g)), phase_of(2 * g), &abort_flag, prm.status, 0x202);
+                if (!ok) break;
+                tc_fence_after();
+                for (int t = 0; t < nt; ++t) {
+                    issue_qk(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
+                    mma_commit(bar(S_FULL + t));
+                }
+                mma_commit(bar(KV_EMPTY + slot_of(2 * g)));
+                if (n == 1) mma_commit(bar(Q_EMPTY));
+                for (int j = 0; j < n; ++j, ++g) {
+                    const uint32_t eV = 2 * g + 1, eKn = 2 * g + 2;
+                    const bool more = j + 1 < n;
+                    if (more) {
+                        ok = wait_or_abort(bar(KV_FULL + slot_of(eKn)), phase_of(eKn), &abort_flag, prm.status, 0x203);
                         if (!ok) break;
+                    }
+                    ok = wait_or_abort(bar(KV_FULL + slot_of(eV)), phase_of(eV), &abort_flag, prm.status, 0x204);
+                    if (!ok) break;
+                    for (int t = 0; t < nt; ++t) {
+                        ok = wait_or_abort(bar(P_READY + t), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
+                        if (!ok) break;
+                        ++cP[t];
                         tc_fence_after();
-#pragma unroll
-                        for (int k = 0; k < HD / 16; ++k) {
-                            const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
-                            mma_ss(tmem + TM_S, smem_desc_sw128(sQ + off, 16, 1024),
-                                   smem_desc_sw128(sK + s * TILE_BYTES + off, 16, 1024), IDESC_QK, k > 0);
+                        issue_pv(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, j > 0);
+                        mma_commit(bar(PV_DONE + t));
+                        if (more) {
+                            issue_qk(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
+                            mma_commit(bar(S_FULL + t));
                         }
-                        mma_commit(bar(K_EMPTY + s));
-                        mma_commit(bar(S_FULL));
-                        if (blk + 1 == wi.kv_blocks) mma_commit(bar(Q_EMPTY));
-                        ok = wait_or_abort(bar(P_READY), it & 1, &abort_flag, prm.status, 0x203);
-                        if (!ok) break;
-                        ok = wait_or_abort(bar(V_FULL + s), ph, &abort_flag, prm.status, 0x204);
-                        if (!ok) break;
-                        tc_fence_after();
-#pragma unroll
-                        for (int k = 0; k < BN / 16; ++k) {
-                            mma_ts(tmem + TM_O, tmem + TM_S + k * 8,
-                                   smem_desc_sw128(sV + s * TILE_BYTES + k * 2048, SLAB_BYTES, 1024), IDESC_PV,
-                                   (blk > 0 || k > 0) ? 1u : 0u);
-                        }
-                        mma_commit(bar(V_EMPTY + s));
-                        mma_commit(bar(O_DONE));
+                    }
+                    if (!ok) break;
+                    mma_commit(bar(KV_EMPTY + slot_of(eV)));
+                    if (more) {
+                        mma_commit(bar(KV_EMPTY + slot_of(eKn)));
+                        if (j + 2 == n) mma_commit(bar(Q_EMPTY));
                     }
                 }
             }
             // every MMA issued above has retired before TMEM is released
             mma_commit(bar(DRAIN));
-            wait_or_abort(bar(DRAIN), 0, &abort_flag, prm.status, 0x205);
+            wait_or_abort(bar(DRAIN), 0, &abort_flag, prm.status, 0x207);
         }
-    } else {
-        // ------------------------------------------- softmax / correction / epilogue
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        uint32_t it = 0, ocount = 0;
+    } else if (warp < 8) {
+        // ------------------------------------------------- softmax + epilogue, tile t
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        const int t = warp >> 2;
+        const int r = tid & 127;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_addr + t * BN;
+        const uint32_t tO = tmem + lane_addr + 256 + t * HD;
+        const float scale_log2 = prm.scale_log2;
+        uint32_t cS = 0, cPV = 0;
         bool ok = true;
         for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
             const WorkItem wi = prm.work[w / prm.bh];
+            if (wi.q_rows <= t * BM) continue;  // this tile is absent from the item
             const int bh = (int)(w % prm.bh);
             const int b = bh / prm.heads, h = bh % prm.heads;
-            float m = -INFINITY, l = 0.f;
-            int blk = 0;
+            float m_ref = 0.f, l = 0.f;
+            bool first = true;
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                 const int nb = item_blocks(wi, seg);
-                for (int j = 0; j < nb; ++j, ++it, ++blk) {
+                for (int j = 0; j < nb; ++j) {
                     const int valid = min(BN, wi.seg_len[seg] - j * BN);
-                    ok = wait_or_abort(bar(S_FULL), it & 1, &abort_flag, prm.status, 0x301);
+                    ok = wait_or_abort(bar(S_FULL + t), cS & 1, &abort_flag, prm.status, 0x301 + t);
                     if (!ok) break;
+                    ++cS;
                     tc_fence_after();
-                    float s[BN];
+                    uint32_t s[BN];
 #pragma unroll
-                    for (int c = 0; c < BN / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + lane_addr + TM_S + c * 32, r);
-                        tmem_wait_ld();
+                    for (int c = 0; c < BN / 32; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+                    tmem_wait_ld();
+                    if (valid < BN) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
+                        for (int i = 0; i < BN; ++i)
+                            if (i >= valid) s[i] = 0xff800000u;  // -inf
                     }
-                    float mx = -INFINITY;
+                    float mx = __uint_as_float(s[0]);
 #pragma unroll
-                    for (int i = 0; i < BN; ++i) {
-                        s[i] = (i < valid) ? s[i] * prm.scale_log2 : -INFINITY;
-                        mx = fmaxf(mx, s[i]);
-                    }
-                    const float m_new = fmaxf(m, mx);
-                    const float alpha = exp2f(m - m_new);
-                    float sum = 0.f;
-                    uint32_t pk[BN / 2];
-#pragma unroll
-                    for (int i = 0; i < BN; i += 2) {
-                        const float p0 = exp2f(s[i] - m_new), p1 = exp2f(s[i + 1] - m_new);
-                        sum += p0 + p1;
-                        __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-                        pk[i >> 1] = *reinterpret_cast<uint32_t *>(&hh);
-                    }
-                    l = l * alpha + sum;
-                    m = m_new;
-                    if (blk > 0) {
-                        // O accumulated so far belongs to the old maximum
-                        ok = wait_or_abort(bar(O_DONE), ocount & 1, &abort_flag, prm.status, 0x302);
+                    for (int i = 1; i < BN; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
+                    mx *= scale_log2;
+                    if (first) {
+                        m_ref = mx;
+                        first = false;
+                    } else if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
+                        // the accumulator of the blocks so far belongs to the old reference
+                        ok = wait_or_abort(bar(PV_DONE + t), (cPV - 1) & 1, &abort_flag, prm.status, 0x303 + t);
                         if (!ok) break;
-                        ++ocount;
                         tc_fence_after();
+                        const float m_new = fmaxf(m_ref, mx);
+                        const float alpha = ex2(m_ref - m_new);
+                        m_ref = m_new;
+                        l *= alpha;
 #pragma unroll
                         for (int c = 0; c < HD / 32; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(tmem + lane_addr + TM_O + c * 32, r);
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                            tmem_st32(tmem + lane_addr + TM_O + c * 32, r);
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(tO + c * 32, o);
                         }
                     }
+                    const float neg_m = -m_ref;
+                    float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
-                    for (int c = 0; c < BN / 64; ++c) {
-                        uint32_t r[32];
+                    for (int c = 0; c < BN / 32; ++c) {
+                        uint32_t pk[16];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = pk[c * 32 + i];
-                        tmem_st32(tmem + lane_addr + TM_S + c * 32, r);
+                        for (int i = 0; i < 16; ++i) {
+                            const float p0 = ex2(fmaf(__uint_as_float(s[c * 32 + 2 * i]), scale_log2, neg_m));
+                            const float p1 = ex2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), scale_log2, neg_m));
+                            pk[i] = pack_bf16(p0, p1);
+                            // the row sum uses the bf16-rounded weights the MMA will see, so
+                            // numerator and denominator round together
+                            sum0 += __uint_as_float(pk[i] << 16);
+                            sum1 += __uint_as_float(pk[i] & 0xffff0000u);
+                        }
+                        tmem_st16(tS + c * 16, pk);
                     }
+                    l += sum0 + sum1;
                     tmem_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar(P_READY));
+                    mbar_arrive(bar(P_READY + t));
+                    ++cPV;
                 }
             }
             if (!ok) break;
-            // epilogue: O / l -> bf16 -> global, rows beyond the item are dropped
-            ok = wait_or_abort(bar(O_DONE), ocount & 1, &abort_flag, prm.status, 0x303);
+            // epilogue: O / l -> bf16 -> global; rows beyond the item are dropped
+            ok = wait_or_abort(bar(PV_DONE + t), (cPV - 1) & 1, &abort_flag, prm.status, 0x305 + t);
             if (!ok) break;
-            ++ocount;
             tc_fence_after();
             const float inv = 1.f / l;
+            const int row = t * BM + r;
             __nv_bfloat16 *orow = prm.out + (long long)b * prm.stride_b + (long long)h * prm.stride_h +
-                                  (long long)(wi.q_start + tid) * prm.stride_s;
+                                  (long long)(wi.q_start + row) * prm.stride_s;
 #pragma unroll
             for (int c = 0; c < HD / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_addr + TM_O + c * 32, r);
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
-                if (tid < wi.q_rows) {
+                if (row < wi.q_rows) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
-                        uint32_t o4[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * u]) * inv,
-                                                                      __uint_as_float(r[i + 2 * u + 1]) * inv);
-                            o4[u] = *reinterpret_cast<uint32_t *>(&hh);
-                        }
-                        *reinterpret_cast<uint4 *>(orow + c * 32 + i) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                        uint4 pk4;
+                        pk4.x = pack_bf16(__uint_as_float(o[i + 0]) * inv, __uint_as_float(o[i + 1]) * inv);
+                        pk4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                        pk4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                        pk4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + c * 32 + i) = pk4;
                     }
                 }
             }
@@ -313,7 +382,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
     }
@@ -357,10 +426,10 @@ int make_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p) {
 
 void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, const int *seg_start,
                const int *seg_len) {
-    for (int r = 0; r < rows; r += BM) {
+    for (int r = 0; r < rows; r += ITEM_ROWS) {
         WorkItem it{};
         it.q_start = row0 + r;
-        it.q_rows = std::min(BM, rows - r);
+        it.q_rows = std::min(ITEM_ROWS, rows - r);
         it.n_seg = 0;
         it.kv_blocks = 0;
         for (int s = 0; s < n_seg; ++s) {
@@ -390,8 +459,11 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
         if (w.seg0_len > 0) add_items(items, w.seg0_start, w.seg0_len, 3, st, ln);
         if (w.seg1_len > 0) add_items(items, w.seg1_start, w.seg1_len, 3, st, ln);
     }
-    std::stable_sort(items.begin(), items.end(),
-                     [](const WorkItem &a, const WorkItem &b) { return a.kv_blocks > b.kv_blocks; });
+    std::stable_sort(items.begin(), items.end(), [](const WorkItem &a, const WorkItem &b) {
+        const long long ca = (long long)a.kv_blocks * (a.q_rows > BM ? 2 : 1);
+        const long long cb = (long long)b.kv_blocks * (b.q_rows > BM ? 2 : 1);
+        return ca > cb;
+    });
     cudaFree(p->d_work);
     p->d_work = nullptr;
     p->n_work = (int)items.size();
