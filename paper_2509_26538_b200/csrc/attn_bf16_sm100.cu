@@ -26,7 +26,10 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <functional>
 #include <mutex>
+#include <queue>
+#include <utility>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -59,8 +62,8 @@ enum Bar {
 
 struct Params {
     const WorkItem *work;
-    int n_work;
-    int bh;      // batch * heads
+    const WorkUnit *units;   // (item, batch*heads index), grouped by CTA
+    const int *cta_begin;    // [gridDim.x + 1] offsets into units
     int heads;
     long long stride_b, stride_h, stride_s;  // elements
     __nv_bfloat16 *out;
@@ -154,7 +157,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const long long total = (long long)prm.n_work * prm.bh;
+    const int u_begin = prm.cta_begin[blockIdx.x], u_end = prm.cta_begin[blockIdx.x + 1];
 
     // registers move from the data-movement warpgroup to the two softmax warpgroups
     if (warp >= 8) {
@@ -168,9 +171,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             prefetch_tmap(&tmV);
             uint32_t kvc = 0, qc = 0;
             bool ok = true;
-            for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const WorkItem wi = prm.work[w / prm.bh];
-                const int bh = (int)(w % prm.bh);
+            for (int u = u_begin; ok && u < u_end; ++u) {
+                const WorkUnit unit = prm.units[u];
+                const WorkItem wi = prm.work[unit.item];
+                const int bh = unit.bh;
                 const int b = bh / prm.heads, h = bh % prm.heads;
                 const int nt = wi.q_rows > BM ? 2 : 1;
                 ok = wait_or_abort(bar(Q_EMPTY), (qc & 1) ^ 1, &abort_flag, prm.status, 0x101);
@@ -215,8 +219,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool ok = true;
             auto slot_of = [](uint32_t e) { return e % NSTAGE; };
             auto phase_of = [](uint32_t e) { return (e / NSTAGE) & 1; };
-            for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const WorkItem wi = prm.work[w / prm.bh];
+            for (int u = u_begin; ok && u < u_end; ++u) {
+                const WorkItem wi = prm.work[prm.units[u].item];
                 const int nt = wi.q_rows > BM ? 2 : 1;
                 const int n = wi.kv_blocks;
                 ok = wait_or_abort(bar(Q_FULL), qc & 1, &abort_flag, prm.status, 0x201);
@@ -276,10 +280,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const float scale_log2 = prm.scale_log2;
         uint32_t cS = 0, cPV = 0;
         bool ok = true;
-        for (long long w = blockIdx.x; ok && w < total; w += gridDim.x) {
-            const WorkItem wi = prm.work[w / prm.bh];
+        for (int u = u_begin; ok && u < u_end; ++u) {
+            const WorkUnit unit = prm.units[u];
+            const WorkItem wi = prm.work[unit.item];
             if (wi.q_rows <= t * BM) continue;  // this tile is absent from the item
-            const int bh = (int)(w % prm.bh);
+            const int bh = unit.bh;
             const int b = bh / prm.heads, h = bh % prm.heads;
             float m_ref = 0.f, l = 0.f;
             bool first = true;
@@ -300,9 +305,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         for (int i = 0; i < BN; ++i)
                             if (i >= valid) s[i] = 0xff800000u;  // -inf
                     }
-                    float mx = __uint_as_float(s[0]);
+                    // eight independent max chains, then a short tree
+                    float mxa[8];
 #pragma unroll
-                    for (int i = 1; i < BN; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
+                    for (int i = 0; i < 8; ++i) mxa[i] = __uint_as_float(s[i]);
+#pragma unroll
+                    for (int i = 8; i < BN; ++i) mxa[i & 7] = fmaxf(mxa[i & 7], __uint_as_float(s[i]));
+                    float mx = fmaxf(fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])),
+                                     fmaxf(fmaxf(mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
                     mx *= scale_log2;
                     if (first) {
                         m_ref = mx;
@@ -327,7 +337,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         }
                     }
                     const float neg_m = -m_ref;
-                    float sum0 = 0.f, sum1 = 0.f;
+                    float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int c = 0; c < BN / 32; ++c) {
                         uint32_t pk[16];
@@ -338,12 +348,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                             pk[i] = pack_bf16(p0, p1);
                             // the row sum uses the bf16-rounded weights the MMA will see, so
                             // numerator and denominator round together
-                            sum0 += __uint_as_float(pk[i] << 16);
-                            sum1 += __uint_as_float(pk[i] & 0xffff0000u);
+                            sum[(2 * i) & 7] += __uint_as_float(pk[i] << 16);
+                            sum[(2 * i + 1) & 7] += __uint_as_float(pk[i] & 0xffff0000u);
                         }
                         tmem_st16(tS + c * 16, pk);
                     }
-                    l += sum0 + sum1;
+                    l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(bar(P_READY + t));
@@ -465,11 +475,49 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
         return ca > cb;
     });
     cudaFree(p->d_work);
+    cudaFree(p->d_units);
+    cudaFree(p->d_cta_begin);
     p->d_work = nullptr;
+    p->d_units = nullptr;
+    p->d_cta_begin = nullptr;
     p->n_work = (int)items.size();
+    p->n_cta = 0;
     if (items.empty()) return HILBERTA_OK;
+
+    // Static schedule: every (item, batch*head) unit goes to the least-loaded CTA,
+    // longest units first.  Cost = MMA block pairs + a fixed per-unit overhead.
+    const int bh = p->batch * p->heads;
+    const long long n_units = (long long)items.size() * bh;
+    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    const int n_cta = (int)std::min<long long>(n_units, p->sm_count);
+    std::vector<std::vector<WorkUnit>> bins(n_cta);
+    typedef std::pair<long long, int> Load;  // (load, cta)
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
+    for (int i = 0; i < (int)items.size(); ++i) {
+        const long long cost = (long long)items[i].kv_blocks * (items[i].q_rows > BM ? 2 : 1) + 2;
+        for (int j = 0; j < bh; ++j) {
+            Load top = heap.top();
+            heap.pop();
+            bins[top.second].push_back(WorkUnit{i, j});
+            heap.push(Load(top.first + cost, top.second));
+        }
+    }
+    std::vector<WorkUnit> units;
+    std::vector<int> cta_begin(n_cta + 1, 0);
+    units.reserve((size_t)n_units);
+    for (int c = 0; c < n_cta; ++c) {
+        cta_begin[c] = (int)units.size();
+        units.insert(units.end(), bins[c].begin(), bins[c].end());
+    }
+    cta_begin[n_cta] = (int)units.size();
+    p->n_cta = n_cta;
     HB_CUDA(cudaMalloc(&p->d_work, sizeof(WorkItem) * items.size()));
     HB_CUDA(cudaMemcpy(p->d_work, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
+    HB_CUDA(cudaMalloc(&p->d_units, sizeof(WorkUnit) * units.size()));
+    HB_CUDA(cudaMemcpy(p->d_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
+    HB_CUDA(cudaMalloc(&p->d_cta_begin, sizeof(int) * cta_begin.size()));
+    HB_CUDA(cudaMemcpy(p->d_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
@@ -489,8 +537,8 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     if ((rc = make_map(&mv, v, p)) != HILBERTA_OK) return rc;
     Params prm;
     prm.work = p->d_work;
-    prm.n_work = p->n_work;
-    prm.bh = p->batch * p->heads;
+    prm.units = p->d_units;
+    prm.cta_begin = p->d_cta_begin;
     prm.heads = p->heads;
     prm.stride_b = p->stride_b;
     prm.stride_h = p->stride_h;
@@ -498,9 +546,7 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     prm.out = (__nv_bfloat16 *)out;
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.status = p->d_status;
-    const long long total = (long long)p->n_work * prm.bh;
-    const int grid = (int)std::min<long long>(total, p->sm_count);
-    attn_bf16_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, prm);
+    attn_bf16_kernel<<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, prm);
     HB_LAUNCHED();
     return HILBERTA_OK;
 }

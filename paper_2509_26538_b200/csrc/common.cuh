@@ -49,6 +49,13 @@ struct WorkItem {
     int kv_blocks;  // sum over ranges of ceil(len / 128)
 };
 
+// A work item applied to one (batch, head).  Units are assigned to CTAs on the
+// host (longest-processing-time-first) and stored grouped by CTA.
+struct WorkUnit {
+    int item;
+    int bh;
+};
+
 }  // namespace hilberta
 
 struct hilberta_plan_s {
@@ -72,6 +79,9 @@ struct hilberta_plan_s {
     float scale;
     hilberta::WorkItem *d_work;
     int n_work;
+    hilberta::WorkUnit *d_units;  // [n_work * batch * heads], grouped by CTA
+    int *d_cta_begin;             // [n_cta + 1]
+    int n_cta;
     int *d_status;  // [4] error word + diagnostics written by bounded waits
     // workspace of hilberta_forward_host
     void *ws;

@@ -158,6 +158,8 @@ static void free_plan(hilberta_plan_t *p) {
     cudaFree(p->d_row_window);
     cudaFree(p->d_windows);
     cudaFree(p->d_work);
+    cudaFree(p->d_units);
+    cudaFree(p->d_cta_begin);
     cudaFree(p->d_status);
     cudaFree(p->ws);
     delete p;
