@@ -52,10 +52,18 @@ constexpr int SMEM_BYTES = (QT + NSTAGE) * TILE_BYTES + 1024;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_CYCLES = 2000000000ll;  // ~1 s: far beyond any legitimate wait
 constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
+#ifndef HB_POLY_MASK
+#define HB_POLY_MASK 0xff  // exponential i of every pair goes to the FMA pipes when (i & MASK) == MASK; 0xff = never (measured: the softmax is issue-bound, so moving work off the MUFU does not pay yet)
+#endif
+#ifndef HB_SPLIT_P
+#define HB_SPLIT_P 1     // hand P to the MMA issuer in two halves
+#endif
 
 enum Bar {
     Q_FULL = 0, Q_EMPTY, DRAIN,
-    S_FULL, P_READY = S_FULL + QT, PV_DONE = P_READY + QT,
+    S_FULL,
+    P_READY = S_FULL + QT,        // [t * 2 + half]: P columns of keys [64 half, +64) written, 128 arrivals
+    PV_DONE = P_READY + 2 * QT,
     KV_FULL = PV_DONE + QT, KV_EMPTY = KV_FULL + NSTAGE,
     NUM_BARS = KV_EMPTY + NSTAGE
 };
@@ -102,6 +110,26 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
+// 2^x on the FMA pipes (no MUFU): x = n + f with n = round(x), f in [-0.5, 0.5];
+// 2^f by a cubic (max relative error 7.8e-5, far below bf16 rounding), 2^n by an
+// exponent add.  Used for a fixed share of the exponentials so that the MUFU unit
+// and the FMA pipes split the work.  x is clamped at -126 (result ~0).
+__device__ __forceinline__ float ex2_poly(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;            // 1.5 * 2^23: the integer lands in the low mantissa bits
+    const float f = x - (t - 12582912.f);
+    float p = fmaf(f, 0.055088773f, 0.24260406f);
+    p = fmaf(p, f, 0.69327623f);
+    p = fmaf(p, f, 0.99992895f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&h);
@@ -110,20 +138,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // S_t = Q_t K^T for one 128-key block: 8 MMAs of K = 16.
 __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t sQt, uint32_t sKslot) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, BN, 0, 0);
+    // the start-address field is the low 14 bits (16-byte units): stepping K is one add
+    const uint64_t dq = smem_desc_sw128(sQt, 16, 1024), dk = smem_desc_sw128(sKslot, 16, 1024);
 #pragma unroll
     for (int k = 0; k < HD / 16; ++k) {
-        const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
-        mma_ss(tmem_s, smem_desc_sw128(sQt + off, 16, 1024), smem_desc_sw128(sKslot + off, 16, 1024), IDESC,
-               k > 0);
+        const uint64_t off = (uint64_t)(((k >> 2) * SLAB_BYTES + (k & 3) * 32) >> 4);
+        mma_ss(tmem_s, dq + off, dk + off, IDESC, k > 0);
     }
 }
 
 // O_t (+)= P_t V for one 128-key block: P from TMEM, V row-major in smem (N-major operand).
-__device__ __forceinline__ void issue_pv(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, bool accumulate) {
+// `half` selects keys [64 half, +64) of the block: four MMAs of K = 16.
+__device__ __forceinline__ void issue_pv_half(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, int half,
+                                              bool accumulate) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
+    const uint64_t dv = smem_desc_sw128(sVslot + half * 8192, SLAB_BYTES, 1024);
 #pragma unroll
-    for (int k = 0; k < BN / 16; ++k) {
-        mma_ts(tmem_o, tmem_p + k * 8, smem_desc_sw128(sVslot + k * 2048, SLAB_BYTES, 1024), IDESC,
+    for (int k = 0; k < 4; ++k) {
+        mma_ts(tmem_o, tmem_p + half * 32 + k * 8, dv + (uint64_t)((k * 2048) >> 4), IDESC,
                (accumulate || k > 0) ? 1u : 0u);
     }
 }
@@ -146,7 +178,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < NUM_BARS; ++i)
-            mbar_init(bar(i), (i >= P_READY && i < P_READY + QT) ? 128 : 1);
+            mbar_init(bar(i), (i >= P_READY && i < P_READY + 2 * QT) ? 128 : 1);
         mbar_fence_init();
     }
     if (warp == 8) {
@@ -246,11 +278,16 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     ok = wait_or_abort(bar(KV_FULL + slot_of(eV)), phase_of(eV), &abort_flag, prm.status, 0x204);
                     if (!ok) break;
                     for (int t = 0; t < nt; ++t) {
-                        ok = wait_or_abort(bar(P_READY + t), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
+                        // P arrives in two halves so the first four MMAs overlap the rest of the softmax
+                        ok = wait_or_abort(bar(P_READY + t * 2), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv_half(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
+                        ok = wait_or_abort(bar(P_READY + t * 2 + 1), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
                         if (!ok) break;
                         ++cP[t];
                         tc_fence_after();
-                        issue_pv(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, j > 0);
+                        issue_pv_half(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
                         mma_commit(bar(PV_DONE + t));
                         if (more) {
                             issue_qk(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
@@ -310,9 +347,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < 8; ++i) mxa[i] = __uint_as_float(s[i]);
 #pragma unroll
-                    for (int i = 8; i < BN; ++i) mxa[i & 7] = fmaxf(mxa[i & 7], __uint_as_float(s[i]));
-                    float mx = fmaxf(fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])),
-                                     fmaxf(fmaxf(mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
+                    for (int i = 8; i < BN; i += 2) {
+                        const int c = (i >> 1) & 7;
+                        mxa[c] = max3(mxa[c], __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+                    }
+                    float mx = max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7]));
                     mx *= scale_log2;
                     if (first) {
                         m_ref = mx;
@@ -343,8 +382,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         uint32_t pk[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            const float p0 = ex2(fmaf(__uint_as_float(s[c * 32 + 2 * i]), scale_log2, neg_m));
-                            const float p1 = ex2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), scale_log2, neg_m));
+                            const float x0 = fmaf(__uint_as_float(s[c * 32 + 2 * i]), scale_log2, neg_m);
+                            const float x1 = fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), scale_log2, neg_m);
+                            const float p0 = ex2(x0);
+                            const float p1 = ((i & HB_POLY_MASK) == HB_POLY_MASK) ? ex2_poly(x1) : ex2(x1);  // a fixed share off the MUFU
                             pk[i] = pack_bf16(p0, p1);
                             // the row sum uses the bf16-rounded weights the MMA will see, so
                             // numerator and denominator round together
@@ -352,11 +393,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                             sum[(2 * i + 1) & 7] += __uint_as_float(pk[i] & 0xffff0000u);
                         }
                         tmem_st16(tS + c * 16, pk);
+                        if (HB_SPLIT_P ? (c & 1) : (c == 3)) {  // keys [64 (c >> 1), +64) are in TMEM
+                            tmem_wait_st();
+                            tc_fence_before();
+                            if (HB_SPLIT_P || c == 3) mbar_arrive(bar(P_READY + t * 2 + (c >> 1)));
+                            if (!HB_SPLIT_P) mbar_arrive(bar(P_READY + t * 2));
+                        }
                     }
                     l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
-                    tmem_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(bar(P_READY + t));
                     ++cPV;
                 }
             }
