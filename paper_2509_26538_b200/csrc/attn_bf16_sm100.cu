@@ -53,7 +53,7 @@ constexpr uint32_t TMEM_COLS = 512;
 constexpr long long WAIT_CYCLES = 2000000000ll;  // ~1 s: far beyond any legitimate wait
 constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 #ifndef HB_POLY_MASK
-#define HB_POLY_MASK 0xff  // exponential i of every pair goes to the FMA pipes when (i & MASK) == MASK; 0xff = never (measured: the softmax is issue-bound, so moving work off the MUFU does not pay yet)
+#define HB_POLY_MASK 3   // pair i of every 16 runs its two exponentials on the FMA pipes when (i & MASK) == MASK (3: one pair in four); 0xff = never
 #endif
 #ifndef HB_SPLIT_P
 #define HB_SPLIT_P 1     // hand P to the MMA issuer in two halves
@@ -128,6 +128,21 @@ __device__ __forceinline__ float ex2_poly(float x) {
     p = fmaf(p, f, 0.69327623f);
     p = fmaf(p, f, 0.99992895f);
     return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
+// The same for a pair of values with packed fp32x2 instructions.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
+    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+    float2 p = __ffma2_rn(f, make_float2(0.055088773f, 0.055088773f), make_float2(0.24260406f, 0.24260406f));
+    p = __ffma2_rn(p, f, make_float2(0.69327623f, 0.69327623f));
+    p = __ffma2_rn(p, f, make_float2(0.99992895f, 0.99992895f));
+    p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
+    p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
+    return p;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -375,22 +390,34 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                             tmem_st32(tO + c * 32, o);
                         }
                     }
-                    const float neg_m = -m_ref;
-                    float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_ref, -m_ref);
+                    float2 sum[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+                    // The row sum is taken over the fp32 weights; the P V MMA sees them rounded
+                    // to bf16.  For the block's largest weight -- the one that dominates a
+                    // near-one-hot row -- the rounding error is added to the sum, so numerator
+                    // and denominator round together where it matters.
+                    {
+                        const float pm = ex2(mx - m_ref);
+                        l += __uint_as_float(pack_bf16(0.f, pm) & 0xffff0000u) - pm;
+                    }
 #pragma unroll
                     for (int c = 0; c < BN / 32; ++c) {
                         uint32_t pk[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            const float x0 = fmaf(__uint_as_float(s[c * 32 + 2 * i]), scale_log2, neg_m);
-                            const float x1 = fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), scale_log2, neg_m);
-                            const float p0 = ex2(x0);
-                            const float p1 = ((i & HB_POLY_MASK) == HB_POLY_MASK) ? ex2_poly(x1) : ex2(x1);  // a fixed share off the MUFU
-                            pk[i] = pack_bf16(p0, p1);
-                            // the row sum uses the bf16-rounded weights the MMA will see, so
-                            // numerator and denominator round together
-                            sum[(2 * i) & 7] += __uint_as_float(pk[i] << 16);
-                            sum[(2 * i + 1) & 7] += __uint_as_float(pk[i] & 0xffff0000u);
+                            // packed fp32x2 arithmetic: one instruction per pair of scores
+                            const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c * 32 + 2 * i]),
+                                                                    __uint_as_float(s[c * 32 + 2 * i + 1])),
+                                                        sc2, nm2);
+                            float2 p;
+                            if ((i & HB_POLY_MASK) == HB_POLY_MASK) {
+                                p = ex2_poly2(x);  // a fixed share of the pairs runs on the FMA pipes
+                            } else {
+                                p.x = ex2(x.x);
+                                p.y = ex2(x.y);
+                            }
+                            pk[i] = pack_bf16(p.x, p.y);
+                            sum[i & 3] = __fadd2_rn(sum[i & 3], p);
                         }
                         tmem_st16(tS + c * 16, pk);
                         if (HB_SPLIT_P ? (c & 1) : (c == 3)) {  // keys [64 (c >> 1), +64) are in TMEM
@@ -400,7 +427,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                             if (!HB_SPLIT_P) mbar_arrive(bar(P_READY + t * 2));
                         }
                     }
-                    l += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+                    {
+                        const float2 sa = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
+                        l += sa.x + sa.y;
+                    }
                     ++cPV;
                 }
             }
