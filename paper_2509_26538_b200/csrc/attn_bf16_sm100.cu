@@ -58,6 +58,9 @@ constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 #ifndef HB_SPLIT_P
 #define HB_SPLIT_P 1     // hand P to the MMA issuer in two halves
 #endif
+#ifndef HB_WARP_ARRIVE
+#define HB_WARP_ARRIVE 0 // 1: one mbarrier arrival per softmax warp (after a warp sync) instead of one per thread; measured equal
+#endif
 
 enum Bar {
     Q_FULL = 0, Q_EMPTY, DRAIN,
@@ -193,7 +196,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < NUM_BARS; ++i)
-            mbar_init(bar(i), (i >= P_READY && i < P_READY + 2 * QT) ? 128 : 1);
+            mbar_init(bar(i), (i >= P_READY && i < P_READY + 2 * QT) ? (HB_WARP_ARRIVE ? 4 : 128) : 1);
         mbar_fence_init();
     }
     if (warp == 8) {
@@ -206,9 +209,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const uint32_t tmem = tmem_slot;
     const int u_begin = prm.cta_begin[blockIdx.x], u_end = prm.cta_begin[blockIdx.x + 1];
 
-    // registers move from the data-movement warpgroup to the two softmax warpgroups
+    // Registers move from the data-movement warpgroup to the two softmax warpgroups.  The split
+    // is tuned: spills in the MMA issuer (fewer than 88) or in the softmax warps (fewer than
+    // 208) both cost more than 5 % of the kernel time.
     if (warp >= 8) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     }
     if (warp == 8) {
         // ------------------------------------------------------------ producer
@@ -264,6 +269,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             uint32_t qc = 0;
             uint32_t cP[QT] = {0, 0};
             bool ok = true;
+#ifdef HB_TIMING
+            long long tm_p = 0, tm_kv = 0, tm_start = clock64();
+#endif
             auto slot_of = [](uint32_t e) { return e % NSTAGE; };
             auto phase_of = [](uint32_t e) { return (e / NSTAGE) & 1; };
             for (int u = u_begin; ok && u < u_end; ++u) {
@@ -286,21 +294,39 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 for (int j = 0; j < n; ++j, ++g) {
                     const uint32_t eV = 2 * g + 1, eKn = 2 * g + 2;
                     const bool more = j + 1 < n;
+#ifdef HB_TIMING
+                    const long long tk0 = clock64();
+#endif
                     if (more) {
                         ok = wait_or_abort(bar(KV_FULL + slot_of(eKn)), phase_of(eKn), &abort_flag, prm.status, 0x203);
                         if (!ok) break;
                     }
                     ok = wait_or_abort(bar(KV_FULL + slot_of(eV)), phase_of(eV), &abort_flag, prm.status, 0x204);
                     if (!ok) break;
+#ifdef HB_TIMING
+                    tm_kv += clock64() - tk0;
+#endif
                     for (int t = 0; t < nt; ++t) {
+#ifdef HB_TIMING
+                        const long long tp0 = clock64();
+#endif
                         // P arrives in two halves so the first four MMAs overlap the rest of the softmax
                         ok = wait_or_abort(bar(P_READY + t * 2), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
                         if (!ok) break;
                         tc_fence_after();
+#ifdef HB_TIMING
+                        tm_p += clock64() - tp0;
+#endif
                         issue_pv_half(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
+#ifdef HB_TIMING
+                        const long long tp1 = clock64();
+#endif
                         ok = wait_or_abort(bar(P_READY + t * 2 + 1), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
                         if (!ok) break;
                         ++cP[t];
+#ifdef HB_TIMING
+                        tm_p += clock64() - tp1;
+#endif
                         tc_fence_after();
                         issue_pv_half(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
                         mma_commit(bar(PV_DONE + t));
@@ -320,10 +346,17 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             // every MMA issued above has retired before TMEM is released
             mma_commit(bar(DRAIN));
             wait_or_abort(bar(DRAIN), 0, &abort_flag, prm.status, 0x207);
+#ifdef HB_TIMING
+            atomicAdd(prm.status + 16, (int)(tm_p >> 4));
+            atomicAdd(prm.status + 17, (int)(tm_kv >> 4));
+            atomicAdd(prm.status + 19, (int)((clock64() - tm_start) >> 4));
+            atomicMax(prm.status + 20, (int)((clock64() - tm_start) >> 4));
+            atomicMin(prm.status + 21, -(int)((clock64() - tm_start) >> 4));
+#endif
         }
     } else if (warp < 8) {
         // ------------------------------------------------- softmax + epilogue, tile t
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int t = warp >> 2;
         const int r = tid & 127;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -332,6 +365,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const float scale_log2 = prm.scale_log2;
         uint32_t cS = 0, cPV = 0;
         bool ok = true;
+#ifdef HB_TIMING
+        long long tm_wait = 0, tm_soft = 0, tm_epi = 0, tm_mark = clock64(), tm_blocks = 0;
+#endif
         for (int u = u_begin; ok && u < u_end; ++u) {
             const WorkUnit unit = prm.units[u];
             const WorkItem wi = prm.work[unit.item];
@@ -347,6 +383,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     ok = wait_or_abort(bar(S_FULL + t), cS & 1, &abort_flag, prm.status, 0x301 + t);
                     if (!ok) break;
                     ++cS;
+#ifdef HB_TIMING
+                    { const long long now = clock64(); tm_wait += now - tm_mark; tm_mark = now; ++tm_blocks; }
+#endif
                     tc_fence_after();
                     uint32_t s[BN];
 #pragma unroll
@@ -423,8 +462,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         if (HB_SPLIT_P ? (c & 1) : (c == 3)) {  // keys [64 (c >> 1), +64) are in TMEM
                             tmem_wait_st();
                             tc_fence_before();
-                            if (HB_SPLIT_P || c == 3) mbar_arrive(bar(P_READY + t * 2 + (c >> 1)));
-                            if (!HB_SPLIT_P) mbar_arrive(bar(P_READY + t * 2));
+                            if (HB_WARP_ARRIVE) __syncwarp();
+                            if (!HB_WARP_ARRIVE || (tid & 31) == 0) {
+                                if (HB_SPLIT_P || c == 3) mbar_arrive(bar(P_READY + t * 2 + (c >> 1)));
+                                if (!HB_SPLIT_P) mbar_arrive(bar(P_READY + t * 2));
+                            }
                         }
                     }
                     {
@@ -432,6 +474,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         l += sa.x + sa.y;
                     }
                     ++cPV;
+#ifdef HB_TIMING
+                    { const long long now = clock64(); tm_soft += now - tm_mark; tm_mark = now; }
+#endif
                 }
             }
             if (!ok) break;
@@ -461,7 +506,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 }
             }
             tc_fence_before();
+#ifdef HB_TIMING
+            { const long long now = clock64(); tm_epi += now - tm_mark; tm_mark = now; }
+#endif
         }
+#ifdef HB_TIMING
+        if ((tid & 127) == 0) {
+            atomicAdd(prm.status + 8 + t * 4 + 0, (int)(tm_wait >> 4));
+            atomicAdd(prm.status + 8 + t * 4 + 1, (int)(tm_soft >> 4));
+            atomicAdd(prm.status + 8 + t * 4 + 2, (int)(tm_epi >> 4));
+            atomicAdd(prm.status + 8 + t * 4 + 3, (int)tm_blocks);
+        }
+#endif
     }
 
     tc_fence_before();
