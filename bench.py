@@ -196,6 +196,9 @@ def main():
     ap.add_argument("--tile", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--schedule", action="store_true",
+                    help="also time the 57-layer per-step schedule (one permute, 57 forwards with the "
+                         "per-layer offsets, one unpermute) on the chosen workload's shape")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -321,6 +324,44 @@ def main():
                "steps": n_e2e}
         assert torch.isfinite(oh.float()).all()
 
+    schedule = None
+    if args.schedule:
+        from paper_2509_26538_b200.inputs import SCHEDULE_LAYERS, schedule_offset
+        offs = [schedule_offset(layer, wl.tile, wl.HW) for layer in range(SCHEDULE_LAYERS)]
+        plans = {}
+        for o in sorted(set(offs)):
+            plans[o] = hb.Plan(wl.H, wl.W, wl.tile, o, wl.shared_region, wl.n_text)
+            plans[o].bind_like(qp)
+        sched_flops = sum(4.0 * wl.head_dim * wl.heads * wl.batch * int(plans[o].export(hb.EXPORT_NNZ)[0])
+                          for o in offs)
+
+        def sched_step():
+            plan.permute(qd, qp)
+            plan.permute(kd, kp)
+            plan.permute(vd, vp)
+            for o in offs:
+                plans[o].forward(qp, kp, vp, op)
+            plan.unpermute(op, od)
+
+        for _ in range(3):
+            sched_step()
+        torch.cuda.synchronize()
+        reps = max(3, min(args.steps, 10))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(reps):
+            sched_step()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        sched_ms = s0.elapsed_time(s1) / reps
+        schedule = {"layers": SCHEDULE_LAYERS, "distinct_plans": len(plans), "ms_per_step": sched_ms,
+                    "ms_per_layer": sched_ms / SCHEDULE_LAYERS, "useful_tflops": sched_flops / (sched_ms * 1e-3) / 1e12,
+                    "offsets": "(layer * tile / 4) mod HW", "reps": reps,
+                    "note": "same Q/K/V for every layer (synthetic); one entry permute of Q, K, V and one exit unpermute"}
+        for p_ in plans.values():
+            assert p_.status() == 0
+            p_.destroy()
+
     if rank != 0:
         if distributed:
             dist.destroy_process_group()
@@ -328,8 +369,9 @@ def main():
 
     peak = peaks["bf16_tflops"]
     line = {
-        "metric": "sparse-attn useful TFLOP/s at 2048^2 (Flux shape)", "value": value, "unit": "TFLOP/s",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "metric": "sparse-attn useful TFLOP/s at %s (Flux shape)" % {"flux1024": "1024^2", "flux2048": "2048^2",
+                                                                      "flux4096": "4096^2"}.get(wl.name, wl.name),
+        "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(wl, world),
         "attn_ms_per_call": fwd_avg, "attn_ms_per_call_median": statistics.median(fwd_ms),
@@ -346,7 +388,7 @@ def main():
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_source": peaks["source"] + " burst",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "traffic": FORWARD_DRAM_TRAFFIC_BYTES.get(wl.name)},
-        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "schedule57": schedule,
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
                              "(4.36 ms per call at 2048^2, 16 tiles)"},
     }
