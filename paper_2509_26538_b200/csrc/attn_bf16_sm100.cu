@@ -79,6 +79,7 @@ struct Params {
     long long stride_b, stride_h, stride_s;  // elements
     __nv_bfloat16 *out;
     float scale_log2;
+    int out_align32;         // out and its strides are 32-byte aligned: 32-byte stores allowed
     int *status;
 };
 
@@ -146,6 +147,12 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
     p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
     p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
     return p;
+}
+
+__device__ __forceinline__ void st_global_v8(void *p, const uint32_t *w) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -494,14 +501,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
                 if (row < wi.q_rows) {
+                    uint32_t w[16];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 pk4;
-                        pk4.x = pack_bf16(__uint_as_float(o[i + 0]) * inv, __uint_as_float(o[i + 1]) * inv);
-                        pk4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-                        pk4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-                        pk4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c * 32 + i) = pk4;
+                    for (int i = 0; i < 16; ++i)
+                        w[i] = pack_bf16(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
+                    if (prm.out_align32) {
+                        // 32-byte stores fill whole sectors: half the store instructions and
+                        // half the L1/L2 write requests of 16-byte stores
+#pragma unroll
+                        for (int i = 0; i < 16; i += 8)
+                            st_global_v8(orow + c * 32 + 2 * i, w + i);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            *reinterpret_cast<uint4 *>(orow + c * 32 + 2 * i) = make_uint4(w[i], w[i + 1], w[i + 2], w[i + 3]);
                     }
                 }
             }
@@ -676,6 +689,7 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     prm.out = (__nv_bfloat16 *)out;
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.status = p->d_status;
+    prm.out_align32 = (((uintptr_t)out & 31) == 0 && ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
     attn_bf16_kernel<<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, prm);
     HB_LAUNCHED();
     return HILBERTA_OK;

@@ -175,8 +175,8 @@ static int build_plan(hilberta_plan_t *p) {
     HB_CUDA(cudaMalloc(&p->d_orig2phys, sizeof(int) * S));
     HB_CUDA(cudaMalloc(&p->d_row_window, sizeof(int) * S));
     HB_CUDA(cudaMalloc(&p->d_windows, sizeof(Window) * p->T));
-    HB_CUDA(cudaMalloc(&p->d_status, sizeof(int) * 64));
-    HB_CUDA(cudaMemset(p->d_status, 0, sizeof(int) * 64));
+    HB_CUDA(cudaMalloc(&p->d_status, sizeof(int) * 4096));
+    HB_CUDA(cudaMemset(p->d_status, 0, sizeof(int) * 4096));
     HB_CUDA(cudaMalloc(&d_shared, HW));
 
     const int sh_lo = p->H / 2 - p->shared_region / 2;
@@ -324,7 +324,7 @@ extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *ho
             hsrc = tmp.data();
             break;
 #ifdef HB_TIMING
-        case 100: need = sizeof(int) * 64; dsrc = p->d_status; break;  // role cycle counters
+        case 100: need = sizeof(int) * 4096; dsrc = p->d_status; break;  // role cycle counters and event trace
 #endif
         default: return HILBERTA_ERR_INVALID;
     }
