@@ -134,6 +134,15 @@ int hilberta_plan_bind(hilberta_plan_t *plan, int batch, int heads, int head_dim
 int hilberta_forward(const void *q, const void *k, const void *v, void *out,
                      const hilberta_plan_t *plan, void *stream);
 
+/* hilberta_forward with the exit gather of Sec. 3.4 fused into its epilogue (the
+ * last attention layer of a step): q, k, v are in PHYSICAL order as for
+ * hilberta_forward; `out` is written in ORIGINAL token order, i.e. physical row p
+ * lands at row phys2orig[p].  Same layout, alignment, error and stream rules as
+ * hilberta_forward.  Costs the same as hilberta_forward (each row is stored by one
+ * thread either way) and saves the separate hilberta_unpermute pass. */
+int hilberta_forward_unpermute(const void *q, const void *k, const void *v, void *out,
+                               const hilberta_plan_t *plan, void *stream);
+
 /* Entry gather of Sec. 3.4 (reordering is one row gather through the Hilbert table):
  *   dst[b, p, :] = src[b, phys2orig[p], :]   for b < batch, p < S.
  * src is in ORIGINAL order, dst in PHYSICAL order; both device pointers to

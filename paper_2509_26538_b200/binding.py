@@ -24,7 +24,8 @@ BF16, FP32 = 0, 1
 # every symbol include/hilberta.h declares
 SYMBOLS = (
     "hilberta_plan", "hilberta_plan_destroy", "hilberta_plan_export", "hilberta_plan_bind",
-    "hilberta_forward", "hilberta_permute", "hilberta_unpermute", "hilberta_forward_host",
+    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_permute", "hilberta_unpermute",
+    "hilberta_forward_host",
     "hilberta_plan_status", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
     "hilberta_last_cuda_error",
 )
@@ -62,6 +63,8 @@ def lib():
     L.hilberta_plan_bind.restype = i32
     L.hilberta_forward.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward.restype = i32
+    L.hilberta_forward_unpermute.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.hilberta_forward_unpermute.restype = i32
     L.hilberta_forward_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_host.restype = i32
     for name in ("hilberta_permute", "hilberta_unpermute"):
@@ -165,6 +168,12 @@ class Plan:
     def forward(self, q, k, v, out, stream=None):
         _check(lib().hilberta_forward(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), self._h,
                                       _stream_ptr(stream)), "hilberta_forward")
+        return out
+
+    def forward_unpermute(self, q, k, v, out, stream=None):
+        """Forward whose output lands in ORIGINAL token order (exit gather fused in)."""
+        _check(lib().hilberta_forward_unpermute(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                                self._h, _stream_ptr(stream)), "hilberta_forward_unpermute")
         return out
 
     def forward_host(self, q, k, v, out, stream=None):

@@ -80,6 +80,7 @@ struct Params {
     __nv_bfloat16 *out;
     float scale_log2;
     int out_align32;         // out and its strides are 32-byte aligned: 32-byte stores allowed
+    const int *out_map;      // nullptr, or physical row -> row of `out` (fused exit scatter)
     int *status;
 };
 
@@ -120,21 +121,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return y;
 }
 
-// 2^x on the FMA pipes (no MUFU): x = n + f with n = round(x), f in [-0.5, 0.5];
-// 2^f by a cubic (max relative error 7.8e-5, far below bf16 rounding), 2^n by an
-// exponent add.  Used for a fixed share of the exponentials so that the MUFU unit
-// and the FMA pipes split the work.  x is clamped at -126 (result ~0).
-__device__ __forceinline__ float ex2_poly(float x) {
-    x = fmaxf(x, -126.f);
-    const float t = x + 12582912.f;            // 1.5 * 2^23: the integer lands in the low mantissa bits
-    const float f = x - (t - 12582912.f);
-    float p = fmaf(f, 0.055088773f, 0.24260406f);
-    p = fmaf(p, f, 0.69327623f);
-    p = fmaf(p, f, 0.99992895f);
-    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
-}
-
-// The same for a pair of values with packed fp32x2 instructions.
+// 2^x for a pair of values on the FMA pipes (no MUFU), with packed fp32x2 instructions:
+// x = n + f with n = round(x) (adding 1.5 * 2^23 leaves the integer in the low mantissa
+// bits), f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.8e-5, far below bf16
+// rounding), 2^n by an exponent add.  Used for a fixed share of the exponentials so that
+// the MUFU unit and the FMA pipes split the work.  x is clamped at -126 (result ~0).
 __device__ __forceinline__ float2 ex2_poly2(float2 x) {
     x.x = fmaxf(x.x, -126.f);
     x.y = fmaxf(x.y, -126.f);
@@ -493,8 +484,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tc_fence_after();
             const float inv = 1.f / l;
             const int row = t * BM + r;
+            // each thread stores its own row, so writing it at its ORIGINAL position instead
+            // of the physical one (the exit gather of Sec. 3.4 fused in) costs one index read
+            int out_row = wi.q_start + row;
+            if (prm.out_map && row < wi.q_rows) out_row = prm.out_map[out_row];
             __nv_bfloat16 *orow = prm.out + (long long)b * prm.stride_b + (long long)h * prm.stride_h +
-                                  (long long)(wi.q_start + row) * prm.stride_s;
+                                  (long long)out_row * prm.stride_s;
 #pragma unroll
             for (int c = 0; c < HD / 32; ++c) {
                 uint32_t o[32];
@@ -671,7 +666,7 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
 }
 
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     cudaStream_t stream) {
+                     const int *out_map, cudaStream_t stream) {
     if (p->n_work == 0) return HILBERTA_OK;
     CUtensorMap mq, mk, mv;
     int rc;
@@ -689,6 +684,7 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     prm.out = (__nv_bfloat16 *)out;
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.status = p->d_status;
+    prm.out_map = out_map;
     prm.out_align32 = (((uintptr_t)out & 31) == 0 && ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
     attn_bf16_kernel<<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, prm);
     HB_LAUNCHED();
@@ -728,11 +724,10 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
         int rc = hilberta_permute(in[i], perm[i], p, bh, p->head_dim, p->dtype, st);
         if (rc != HILBERTA_OK) return rc;
     }
-    int rc = hilberta_forward(perm[0], perm[1], perm[2], out_phys, p, st);
+    (void)bh;
+    int rc = hilberta_forward_unpermute(perm[0], perm[1], perm[2], out_phys, p, st);  // out_phys holds ORIGINAL order
     if (rc != HILBERTA_OK) return rc;
-    rc = hilberta_unpermute(out_phys, in[0], p, bh, p->head_dim, p->dtype, st);
-    if (rc != HILBERTA_OK) return rc;
-    HB_CUDA(cudaMemcpyAsync(out, in[0], bytes, cudaMemcpyDeviceToHost, st));
+    HB_CUDA(cudaMemcpyAsync(out, out_phys, bytes, cudaMemcpyDeviceToHost, st));
     HB_CUDA(cudaStreamSynchronize(st));
     return HILBERTA_OK;
 }

@@ -163,3 +163,25 @@ def test_full_size_sampled_rows(name, n_rows):
     ref = oracle_rows(wl.H, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text, q, k, v, rows=rows)
     check(got[:, :, rows], ref)
     assert torch.isfinite(got.float()).all()
+
+
+def test_forward_unpermute_equals_forward_then_unpermute():
+    """The fused exit scatter writes exactly what forward + hilberta_unpermute write."""
+    for (H, tile, o, hs, nt, dtype) in [(32, 256, 128, 4, 77, torch.bfloat16), (16, 64, 16, 2, 5, torch.float32)]:
+        S = nt + H * H
+        D = 128 if dtype == torch.bfloat16 else 64
+        g = torch.Generator().manual_seed(321)
+        q, k, v = (torch.randn((2, 3, S, D), generator=g).to(dtype).cuda() for _ in range(3))
+        plan = hb.Plan(H, H, tile, o, hs, nt)
+        try:
+            plan.bind_like(q)
+            out_phys, out_a = torch.empty_like(q), torch.empty_like(q)
+            out_b = torch.full_like(q, float("nan"))
+            plan.forward(q, k, v, out_phys)
+            plan.unpermute(out_phys, out_a)
+            plan.forward_unpermute(q, k, v, out_b)
+            assert plan.status() == 0
+            view = torch.int16 if dtype == torch.bfloat16 else torch.int32
+            assert torch.equal(out_a.view(view), out_b.view(view))
+        finally:
+            plan.destroy()
