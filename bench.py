@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one forward launch, from the
-# ncu capture summarised in profiles/attn_bf16_kernel_flux2048.md (558.5 MB read + 90.1 MB written).
-FORWARD_DRAM_TRAFFIC_BYTES = {"flux2048": 648.7e6}
+# ncu capture summarised in profiles/attn_bf16_kernel_flux2048.md (555.1 MB read + 92.4 MB written).
+FORWARD_DRAM_TRAFFIC_BYTES = {"flux2048": 647.5e6}
 
 
 def load_peaks():

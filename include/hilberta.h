@@ -134,6 +134,15 @@ int hilberta_plan_bind(hilberta_plan_t *plan, int batch, int heads, int head_dim
 int hilberta_forward(const void *q, const void *k, const void *v, void *out,
                      const hilberta_plan_t *plan, void *stream);
 
+/* hilberta_forward that also returns the log-sum-exp of every query row (the
+ * max-logits buffer M of Algorithm 1, final step "m + log l"), as a backward pass
+ * would need it.  lse: device pointer to [batch * heads, S] fp32, PHYSICAL row
+ * order, natural logarithm of the sum over kept keys of exp(scale * <q, k>).
+ * Everything else as hilberta_forward.  (Algorithm 1 stores the base-2 value of
+ * the scaled logits; multiply by log2(e) to get it.) */
+int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out, float *lse,
+                         const hilberta_plan_t *plan, void *stream);
+
 /* hilberta_forward with the exit gather of Sec. 3.4 fused into its epilogue (the
  * last attention layer of a step): q, k, v are in PHYSICAL order as for
  * hilberta_forward; `out` is written in ORIGINAL token order, i.e. physical row p

@@ -24,7 +24,8 @@ BF16, FP32 = 0, 1
 # every symbol include/hilberta.h declares
 SYMBOLS = (
     "hilberta_plan", "hilberta_plan_destroy", "hilberta_plan_export", "hilberta_plan_bind",
-    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_permute", "hilberta_unpermute",
+    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_lse", "hilberta_permute",
+    "hilberta_unpermute",
     "hilberta_forward_host",
     "hilberta_plan_status", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
     "hilberta_last_cuda_error",
@@ -65,6 +66,8 @@ def lib():
     L.hilberta_forward.restype = i32
     L.hilberta_forward_unpermute.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_unpermute.restype = i32
+    L.hilberta_forward_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.hilberta_forward_lse.restype = i32
     L.hilberta_forward_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_host.restype = i32
     for name in ("hilberta_permute", "hilberta_unpermute"):
@@ -175,6 +178,12 @@ class Plan:
         _check(lib().hilberta_forward_unpermute(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                                 self._h, _stream_ptr(stream)), "hilberta_forward_unpermute")
         return out
+
+    def forward_lse(self, q, k, v, out, lse, stream=None):
+        """Forward that also writes the per-row log-sum-exp (fp32 [B, heads, S], physical order)."""
+        _check(lib().hilberta_forward_lse(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                          lse.data_ptr(), self._h, _stream_ptr(stream)), "hilberta_forward_lse")
+        return out, lse
 
     def forward_host(self, q, k, v, out, stream=None):
         """q, k, v, out: HOST tensors (pinned for asynchronous copies), original order."""

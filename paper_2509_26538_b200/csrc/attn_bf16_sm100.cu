@@ -81,6 +81,8 @@ struct Params {
     float scale_log2;
     int out_align32;         // out and its strides are 32-byte aligned: 32-byte stores allowed
     const int *out_map;      // nullptr, or physical row -> row of `out` (fused exit scatter)
+    float *lse;              // nullptr, or [batch * heads, S] log-sum-exp (natural log), rows as `out`
+    int S;
     int *status;
 };
 
@@ -490,6 +492,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (prm.out_map && row < wi.q_rows) out_row = prm.out_map[out_row];
             __nv_bfloat16 *orow = prm.out + (long long)b * prm.stride_b + (long long)h * prm.stride_h +
                                   (long long)out_row * prm.stride_s;
+            // m_ref and l are in the base-2 domain of the scaled logits: LSE = ln 2 * (m_ref + log2 l)
+            if (prm.lse && row < wi.q_rows)
+                prm.lse[(long long)bh * prm.S + out_row] = 0.6931471805599453f * (m_ref + log2f(l));
 #pragma unroll
             for (int c = 0; c < HD / 32; ++c) {
                 uint32_t o[32];
@@ -666,7 +671,7 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
 }
 
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     const int *out_map, cudaStream_t stream) {
+                     float *lse, const int *out_map, cudaStream_t stream) {
     if (p->n_work == 0) return HILBERTA_OK;
     CUtensorMap mq, mk, mv;
     int rc;
@@ -685,6 +690,8 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.status = p->d_status;
     prm.out_map = out_map;
+    prm.lse = lse;
+    prm.S = p->S;
     prm.out_align32 = (((uintptr_t)out & 31) == 0 && ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
     attn_bf16_kernel<<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, prm);
     HB_LAUNCHED();

@@ -17,7 +17,8 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32)
 attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
                  float *__restrict__ out, long long stride_b, long long stride_h, long long stride_s,
                  int heads, int S, int P, const int *__restrict__ row_window,
-                 const Window *__restrict__ windows, const int *__restrict__ out_map, float scale) {
+                 const Window *__restrict__ windows, const int *__restrict__ out_map, float *__restrict__ lse,
+                 float scale) {
     __shared__ float sq[kRowsPerBlock][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * kRowsPerBlock + warp;
@@ -104,12 +105,13 @@ attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const
     }
     const int out_row = out_map ? out_map[row] : row;  // optional fused exit scatter
     float *orow = out + base + (long long)out_row * stride_s;
+    if (lse && lane == 0) lse[(long long)bh * S + out_row] = m_all + logf(l);
 #pragma unroll
     for (int i = 0; i < D / 32; ++i) orow[i * 32 + lane] = mine[i];
 }
 
 int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     const int *out_map, cudaStream_t stream) {
+                     float *lse, const int *out_map, cudaStream_t stream) {
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
     if ((bits & 15) || ((p->stride_b | p->stride_h | p->stride_s) & 3)) return HILBERTA_ERR_INVALID;
     dim3 grid((p->S + kRowsPerBlock - 1) / kRowsPerBlock, p->batch * p->heads);
@@ -119,7 +121,7 @@ int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, con
         attn_fp32_kernel<DD><<<grid, block, 0, stream>>>(                                             \
             (const float *)q, (const float *)k, (const float *)v, (float *)out, p->stride_b,          \
             p->stride_h, p->stride_s, p->heads, p->S, p->P, p->d_row_window, p->d_windows, out_map,   \
-            p->scale);                                                                                \
+            lse, p->scale);                                                                                \
         break;
     switch (p->head_dim) {
         HB_FP32_CASE(32)

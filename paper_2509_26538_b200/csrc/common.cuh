@@ -92,9 +92,11 @@ struct hilberta_plan_s {
 namespace hilberta {
 // out_map: nullptr = write rows in physical order; else out_map[p] is the row of `out`
 // that physical row p goes to (the exit gather fused into the epilogue).
+// lse: nullptr, or [batch * heads, S] fp32 receiving log-sum-exp of the scaled logits
+// (natural log), indexed like `out` rows.
 int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     const int *out_map, cudaStream_t stream);
+                     float *lse, const int *out_map, cudaStream_t stream);
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     const int *out_map, cudaStream_t stream);
+                     float *lse, const int *out_map, cudaStream_t stream);
 int attn_bf16_prepare(hilberta_plan_t *p);
 }  // namespace hilberta
