@@ -11,6 +11,9 @@ and in float64.
 
 Where each piece comes from
 ---------------------------
+* padded_side / hilbert_cell_index : general H x W grids (Appendix "Hilbert Curve
+  for General Shape"): the curve of the smallest enclosing power-of-two square,
+  restricted to the real cells; tiles are cut on the padded curve.
 * hilbert_d2t / hilbert_t2d : the bijection pi and its inverse (Sec. 3.1, the
   graph model of the grid and "a bijection pi that visits each cell once").
   The paper names the Hilbert curve but fixes no orientation; the recursion
@@ -68,17 +71,38 @@ def _log2_exact(n: int) -> int:
     return k
 
 
+def padded_side(H: int, W: int) -> int:
+    """Side n = 2^k of the smallest enclosing power-of-two square (Appendix "Hilbert
+    Curve for General Shape": the curve is built on an enclosing regular grid and the
+    H x W sub-region is extracted; cells outside it are padding)."""
+    if H < 1 or W < 1:
+        raise ValueError("empty grid")
+    n = 1
+    while n < max(H, W):
+        n *= 2
+    return n
+
+
+def hilbert_cell_index(H: int, W: int) -> np.ndarray:
+    """row-major cell id r*W + c -> Hilbert index of the cell on the padded n x n grid.
+    int32[HW].  For a power-of-two square this is pi^-1 itself."""
+    n = padded_side(H, W)
+    pts = hilbert_points(_log2_exact(n))
+    out = np.empty(H * W, dtype=np.int32)
+    for d, (x, y) in enumerate(pts):
+        if y < H and x < W:
+            out[y * W + x] = d
+    return out
+
+
 def hilbert_d2t(H: int, W: int) -> np.ndarray:
-    """d -> row-major cell id r*W + c (pi of Sec. 3.1). int32[HW]."""
-    if H != W:
-        raise ValueError("square power-of-two grids only")
-    k = _log2_exact(H)
-    pts = hilbert_points(k)
-    return np.array([y * W + x for (x, y) in pts], dtype=np.int32)
+    """d -> row-major cell id r*W + c (pi of Sec. 3.1). int32[HW].  On a general
+    shape d is the RANK of the cell among the real cells in padded-curve order."""
+    return np.argsort(hilbert_cell_index(H, W), kind="stable").astype(np.int32)
 
 
 def hilbert_t2d(H: int, W: int) -> np.ndarray:
-    """row-major cell id -> Hilbert index d (pi^-1). int32[HW]."""
+    """row-major cell id -> Hilbert index d (pi^-1; rank on a general shape). int32[HW]."""
     d2t = hilbert_d2t(H, W)
     t2d = np.empty_like(d2t)
     t2d[d2t] = np.arange(d2t.size, dtype=np.int32)
@@ -104,9 +128,9 @@ def shared_cells(H: int, W: int, shared_region: int) -> np.ndarray:
 
 
 def shared_hilbert_indices(H: int, W: int, shared_region: int) -> np.ndarray:
-    """Sorted Hilbert indices of the shared cells."""
-    t2d = hilbert_t2d(H, W)
-    return np.sort(t2d[shared_cells(H, W, shared_region)]).astype(np.int32)
+    """Sorted (padded) Hilbert indices of the shared cells."""
+    pidx = hilbert_cell_index(H, W)
+    return np.sort(pidx[shared_cells(H, W, shared_region)]).astype(np.int32)
 
 
 # --------------------------------------------------------------------------
@@ -128,15 +152,19 @@ def token_classes(H, W, tile, layer_offset, shared_region, n_text):
 
     Text tokens and shared-region tokens are global (Appendix A / Sec. 3.3);
     every image token, shared or not, has a tile id from its Hilbert index.
+    On a general shape the tiles are cut on the padded curve (padding positions
+    stay in the sequence and are masked out, as the appendix says), so `tile`
+    must divide the padded length n*n.
     """
     HW = H * W
     S = n_text + HW
-    t2d = hilbert_t2d(H, W)
+    n = padded_side(H, W)
+    pidx = hilbert_cell_index(H, W)
     is_global = np.zeros(S, dtype=np.uint8)
     is_global[:n_text] = 1
     is_global[n_text + shared_cells(H, W, shared_region)] = 1
     group = np.full(S, -1, dtype=np.int32)
-    group[n_text:] = group_of(t2d, layer_offset, HW, tile).astype(np.int32)
+    group[n_text:] = group_of(pidx, layer_offset, n * n, tile).astype(np.int32)
     return is_global, group
 
 
@@ -166,7 +194,7 @@ def nnz(H, W, tile, layer_offset, shared_region, n_text) -> int:
     S = is_global.size
     n_global = int(is_global.sum())
     nonshared_img = (group >= 0) & (is_global == 0)
-    T = (H * W) // tile
+    T = (padded_side(H, W) ** 2) // tile
     per_group = np.bincount(group[nonshared_img], minlength=T).astype(np.int64)
     total = n_global * S
     # a non-global row sees every global column plus the non-global members of its tile
@@ -240,31 +268,38 @@ def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
     non-shared image tokens by ascending Hilbert index].
 
     windows[w] = (lo, seg0_start, seg0_len, seg1_start, seg1_len): tile w of
-    the slid partition covers Hilbert indices [lo, lo + tile) modulo HW; its
-    non-shared members occupy one or (if it wraps) two contiguous physical
-    ranges.  seg0 is the range that starts at lo.  Empty ranges are (0, 0).
+    the slid partition covers (padded) Hilbert indices [lo, lo + tile) modulo
+    n*n; its non-shared real members occupy one or (if it wraps) two contiguous
+    physical ranges.  seg0 is the range that starts at lo.  Empty ranges are (0, 0).
+    shared_runs are maximal runs of shared (padded) Hilbert indices.
     """
     HW = H * W
     S = n_text + HW
-    T = HW // tile
-    if tile < 1 or HW % tile:
-        raise ValueError("tile must divide H*W")
+    n = padded_side(H, W)
+    NP = n * n
+    if tile < 1 or NP % tile:
+        raise ValueError("tile must divide the (padded) curve length")
+    T = NP // tile
     d2t = hilbert_d2t(H, W)
     t2d = hilbert_t2d(H, W)
-    sh = shared_hilbert_indices(H, W, shared_region)
+    pidx = hilbert_cell_index(H, W)                      # cell -> padded index
+    sh_cells = shared_cells(H, W, shared_region)
+    sh = np.sort(pidx[sh_cells]).astype(np.int32)        # shared padded indices
     n_sh = sh.size
     P = n_text + n_sh
-    is_sh = np.zeros(HW, dtype=bool)
+    cell_of = np.full(NP, -1, dtype=np.int64)            # padded index -> cell or -1 (padding)
+    cell_of[pidx] = np.arange(HW)
+    is_sh = np.zeros(NP, dtype=bool)
     is_sh[sh] = True
+    real_ns = (cell_of >= 0) & ~is_sh                    # real, non-shared, by padded index
 
     phys2orig = np.empty(S, dtype=np.int32)
     phys2orig[:n_text] = np.arange(n_text)
-    phys2orig[n_text:P] = n_text + d2t[sh]
-    phys2orig[P:] = n_text + d2t[~is_sh]
+    phys2orig[n_text:P] = n_text + cell_of[sh]
+    phys2orig[P:] = n_text + cell_of[real_ns]
     orig2phys = np.empty(S, dtype=np.int32)
     orig2phys[phys2orig] = np.arange(S, dtype=np.int32)
 
-    # maximal runs of consecutive shared Hilbert indices
     runs = []
     for d in sh.tolist():
         if runs and runs[-1][0] + runs[-1][1] == d:
@@ -273,21 +308,21 @@ def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
             runs.append([d, 1])
     shared_runs = np.array(runs, dtype=np.int32).reshape(-1, 2)
 
-    # c[d] = number of non-shared Hilbert indices below d, d in [0, HW]
-    c = np.concatenate([[0], np.cumsum(~is_sh)]).astype(np.int64)
-    o = int(layer_offset) % HW
+    # c[d] = number of real non-shared cells with padded index below d, d in [0, NP]
+    c = np.concatenate([[0], np.cumsum(real_ns)]).astype(np.int64)
+    o = int(layer_offset) % NP
     windows = np.zeros((T, 5), dtype=np.int32)
     for w in range(T):
-        lo = (w * tile - o) % HW
+        lo = (w * tile - o) % NP
         hi = lo + tile
-        if hi <= HW:
+        if hi <= NP:
             segs = [(lo, hi)]
         else:
-            segs = [(lo, HW), (0, hi - HW)]
+            segs = [(lo, NP), (0, hi - NP)]
         row = [lo]
         for (a, b) in segs:
-            n = int(c[b] - c[a])
-            row += [int(P + c[a]), n] if n > 0 else [0, 0]
+            cnt = int(c[b] - c[a])
+            row += [int(P + c[a]), cnt] if cnt > 0 else [0, 0]
         row += [0, 0] * (2 - len(segs))
         windows[w] = row
     return {
@@ -300,6 +335,7 @@ def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
         "nnz": nnz(H, W, tile, layer_offset, shared_region, n_text),
         "n_shared": int(n_sh),
         "prefix": int(P),
+        "padded_side": int(n),
     }
 
 

@@ -113,8 +113,37 @@ def test_worked_points_16():
     assert got == {64: (8, 0), 128: (8, 8), 192: (7, 15), 255: (0, 15)}
 
 
-def test_rejects_bad_grids():
+@pytest.mark.parametrize("H,W", [(6, 6), (8, 16), (3, 5), (7, 2), (1, 9), (12, 20), (5, 5)])
+def test_general_shapes_are_the_padded_curve_restricted(H, W):
+    """Appendix (general shape): the curve of the enclosing power-of-two square,
+    with the cells outside the H x W region dropped and the order kept."""
+    n = orc.padded_side(H, W)
+    assert n >= max(H, W) and n // 2 < max(H, W) and n & (n - 1) == 0
+    k = n.bit_length() - 1
+    pidx = orc.hilbert_cell_index(H, W)
+    # independent construction of the padded index of every real cell
+    where = {}
+    for d in range(n * n):
+        x, y = _bitpair_d2xy(k, d)
+        where[(y, x)] = d
+    ref = np.array([where[(r, c)] for r in range(H) for c in range(W)])
+    assert np.array_equal(pidx, ref)
+    d2t, t2d = orc.hilbert_d2t(H, W), orc.hilbert_t2d(H, W)
+    assert sorted(d2t.tolist()) == list(range(H * W))
+    assert np.array_equal(t2d[d2t], np.arange(H * W))
+    # rank order = padded-curve order
+    assert np.all(np.diff(pidx[d2t]) > 0)
+    # the padded curve visits real cells in runs: consecutive ranks whose padded
+    # indices are consecutive are grid neighbours
+    r, c = np.divmod(d2t.astype(np.int64), W)
+    consecutive = np.diff(pidx[d2t]) == 1
+    step = np.abs(np.diff(r)) + np.abs(np.diff(c))
+    assert np.all(step[consecutive] == 1)
+
+
+def test_power_of_two_square_needs_no_padding():
+    for n in (1, 2, 8, 32):
+        assert orc.padded_side(n, n) == n
+        assert np.array_equal(orc.hilbert_cell_index(n, n), orc.hilbert_t2d(n, n))
     with pytest.raises(ValueError):
-        orc.hilbert_d2t(6, 6)
-    with pytest.raises(ValueError):
-        orc.hilbert_d2t(8, 16)
+        orc.padded_side(0, 4)

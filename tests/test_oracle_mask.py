@@ -9,14 +9,17 @@ from oracle import hilberta_oracle as orc
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "table1_gflops.txt")
 
 
-def _naive_mask(H, W, tile, o, hs, n_text):
+def _naive_mask(H, W, tile, o, hs, n_text):  # H x W need not be square or a power of two
     """Second, independent enumeration: loop over all pairs and test the three
     clauses on grid coordinates, finding the Hilbert index by searching the
     curve's point list."""
-    pts = orc.hilbert_points(int(np.log2(H)))
-    index_of = {(y, x): d for d, (x, y) in enumerate(pts)}
+    n = 1
+    while n < max(H, W):
+        n *= 2
+    pts = orc.hilbert_points(int(np.log2(n)))
+    index_of = {(y, x): d for d, (x, y) in enumerate(pts)}   # index on the padded curve
     HW = H * W
-    T = HW // tile
+    T = (n * n) // tile
     S = n_text + HW
     r0, c0 = H // 2 - hs // 2, W // 2 - hs // 2
 
@@ -68,6 +71,34 @@ def test_mask_structure(H, tile, o, hs, n_text):
         assert np.all(M.sum(axis=1) == tile)
         classes = {tuple(np.nonzero(row)[0]) for row in M}
         assert len(classes) == (H * H) // tile
+
+
+@pytest.mark.parametrize("H,W,tile,o,hs,n_text", [
+    (3, 5, 16, 0, 0, 0), (3, 5, 8, 3, 2, 2), (6, 4, 16, 5, 2, 1), (7, 2, 4, 1, 0, 3), (5, 5, 64, 9, 4, 0),
+    (6, 6, 8, 60, 2, 2), (1, 9, 32, 7, 0, 1),
+])
+def test_mask_bruteforce_general_shapes(H, W, tile, o, hs, n_text):
+    """Appendix (general shape): tiles are cut on the padded curve, padding is masked."""
+    M = orc.mask(H, W, tile, o, hs, n_text)
+    assert np.array_equal(M, _naive_mask(H, W, tile, o, hs, n_text))
+    assert np.array_equal(M, M.T) and M.diagonal().all()
+    assert orc.nnz(H, W, tile, o, hs, n_text) == int(M.sum())
+    # layout and key ranges expand to the same mask
+    p = orc.plan_arrays(H, W, tile, o, hs, n_text)
+    S, P = M.shape[0], p["prefix"]
+    p2o = p["phys2orig"]
+    assert sorted(p2o.tolist()) == list(range(S))
+    Mp = np.zeros((S, S), dtype=bool)
+    Mp[:P, :] = True
+    Mp[:, :P] = True
+    covered = np.zeros(S, dtype=int)
+    for (lo, s0, n0, s1, n1) in p["windows"].tolist():
+        idx = list(range(s0, s0 + n0)) + list(range(s1, s1 + n1))
+        covered[idx] += 1
+        Mp[np.ix_(idx, idx)] = True
+    assert np.all(covered[P:] == 1) and np.all(covered[:P] == 0)
+    assert np.array_equal(Mp, M[np.ix_(p2o, p2o)])
+    assert len(p["windows"]) == orc.padded_side(H, W) ** 2 // tile
 
 
 def test_offset_zero_is_block_diagonal_in_hilbert_order():
