@@ -23,7 +23,13 @@
  *     P = n_text + n_shared is the "global prefix" (the paper's N_s).
  *   - Mask: query i may read key j iff i is in the prefix, or j is in the
  *     prefix, or i and j are image tokens whose slid tile ids
- *     floor(((d + layer_offset) mod HW) / tile) agree, d = Hilbert index.
+ *     floor(((d + layer_offset) mod NP) / tile) agree, d = Hilbert index.
+ *   - General H x W grids (appendix "Hilbert Curve for General Shape"): the
+ *     curve is that of the smallest enclosing power-of-two square, side n,
+ *     NP = n*n positions; cells outside H x W are padding that no token occupies.
+ *     d above is the index on that padded curve (so `tile` must divide NP), while
+ *     the exported Hilbert tables and the physical order rank the real cells in
+ *     curve order.  For H = W = 2^k nothing is padded and NP = H*W.
  */
 #ifndef HILBERTA_H_
 #define HILBERTA_H_
@@ -53,14 +59,14 @@ extern "C" {
 #define HILBERTA_FP32 1
 
 /* selectors for hilberta_plan_export */
-#define HILBERTA_EXPORT_HIL_D2T 0     /* int32[HW]   Hilbert index -> row-major cell r*W+c */
-#define HILBERTA_EXPORT_HIL_T2D 1     /* int32[HW]   row-major cell -> Hilbert index */
+#define HILBERTA_EXPORT_HIL_D2T 0     /* int32[HW]   Hilbert rank (curve order among the real cells) -> cell r*W+c */
+#define HILBERTA_EXPORT_HIL_T2D 1     /* int32[HW]   row-major cell -> Hilbert rank */
 #define HILBERTA_EXPORT_PHYS2ORIG 2   /* int32[S]    physical position -> original token */
 #define HILBERTA_EXPORT_ORIG2PHYS 3   /* int32[S]    original token -> physical position */
-#define HILBERTA_EXPORT_SHARED_RUNS 4 /* int32[n][2] maximal runs (start, length) of shared Hilbert indices */
+#define HILBERTA_EXPORT_SHARED_RUNS 4 /* int32[n][2] maximal runs (start, length) of shared positions on the padded curve */
 #define HILBERTA_EXPORT_WINDOWS 5     /* int32[T][5] per slid tile: lo, seg0_start, seg0_len, seg1_start, seg1_len */
 #define HILBERTA_EXPORT_NNZ 6         /* uint64[1]   number of (query, key) pairs the mask keeps */
-#define HILBERTA_EXPORT_INFO 7        /* int32[8]    H, W, tile, offset mod HW, shared_region, n_text, n_shared, T */
+#define HILBERTA_EXPORT_INFO 7        /* int32[9]    H, W, tile, offset mod NP, shared_region, n_text, n_shared, T, padded side n */
 
 typedef struct hilberta_plan_s hilberta_plan_t;
 
@@ -71,13 +77,14 @@ typedef struct hilberta_plan_s hilberta_plan_t;
  * l Delta = layer_offset, wrap-around indexing), Sec. 3.3 (central shared
  * region) and Appendix A (prefix layout).
  *
- *   H, W           image-token grid; must be equal powers of two, 1 <= H <= 1024
- *                  (other shapes: HILBERTA_ERR_UNSUPPORTED).
- *   tile           N_T in tokens; tile >= 1 and (H*W) % tile == 0, else ERR_INVALID.
- *   layer_offset   slide in tokens, any integer; reduced modulo H*W (only its
- *                  value modulo tile changes the mask).
- *   shared_region  side of the centred square shared region in grid cells;
- *                  0 = none; must be even and <= H, else ERR_INVALID.
+ *   H, W           image-token grid, 1 <= H, W <= 1024 (larger: HILBERTA_ERR_UNSUPPORTED).
+ *   tile           N_T in curve positions; tile >= 1 and NP % tile == 0 (NP = H*W for
+ *                  power-of-two squares), else ERR_INVALID.
+ *   layer_offset   slide in curve positions, any integer; reduced modulo NP (only
+ *                  its value modulo tile changes the mask).
+ *   shared_region  side of the centred square shared region in grid cells (rows
+ *                  [H/2 - s/2, H/2 + s/2), columns likewise); 0 = none; must be even
+ *                  and <= min(H, W), else ERR_INVALID.
  *   n_text         number of text tokens (>= 0) placed before the image tokens.
  *   out            receives the plan.  The library owns it; release with
  *                  hilberta_plan_destroy.  All tables live in device memory.

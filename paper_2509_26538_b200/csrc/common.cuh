@@ -60,12 +60,13 @@ struct WorkUnit {
 
 struct hilberta_plan_s {
     int device;
-    int H, W, HW, k_log2;
+    int H, W, HW, k_log2;   // image grid; padded side n = 2^k_log2 >= max(H, W)
+    int NP;                 // n * n: length of the padded Hilbert curve the tiles are cut on
     int tile, offset, shared_region, n_text, n_shared, T, S, P;
     uint64_t nnz;
     // device tables
     int *d_hil_d2t, *d_hil_t2d;      // [HW]
-    int *d_c;                        // [HW + 1] non-shared Hilbert indices below d
+    int *d_c;                        // [NP + 1] real non-shared cells with padded Hilbert index below d
     int *d_phys2orig, *d_orig2phys;  // [S]
     int *d_row_window;               // [S] window id of a physical row, -1 for prefix rows
     hilberta::Window *d_windows;     // [T]

@@ -12,19 +12,23 @@ thread_local int g_last_cuda_error = 0;
 std::atomic<uint64_t> g_launches{0};
 
 // ---------------------------------------------------------------------------
-// Sec. 3.1: grid cell -> Hilbert index, one thread per cell.
+// Sec. 3.1 + appendix on general shapes: one thread per cell of the padded n x n
+// grid (n = 2^k, the smallest power-of-two square that holds the H x W grid).
 // Walk the bit planes of (col, row) from the most significant one down; each
 // plane contributes a quadrant digit and re-orients the remaining sub-square.
-// The orientation (start at row 0 / col 0, end at row 0 / col W-1) is the one
-// the library documents.  Also flags the cells of the central shared square
-// (Sec. 3.3), indexed by Hilbert index.
+// The orientation (start at row 0 / col 0, end at row 0 / col n-1) is the one
+// the library documents.  Every padded index gets a kind: padding (outside
+// H x W), real, or real and inside the central shared square (Sec. 3.3).
 // ---------------------------------------------------------------------------
-__global__ void hilbert_lut_kernel(int k, int *__restrict__ d2t, int *__restrict__ t2d,
-                                   unsigned char *__restrict__ shared_by_d, int sh_lo, int sh_hi) {
+enum : unsigned char { CELL_PAD = 0, CELL_REAL = 1, CELL_SHARED = 2 };
+
+__global__ void hilbert_lut_kernel(int k, int H, int W, int *__restrict__ cell_of_pd,
+                                   int *__restrict__ pd_of_cell, unsigned char *__restrict__ kind_by_pd,
+                                   int sh_r0, int sh_c0, int sh_side) {
     const int n = 1 << k;
-    const int cell = blockIdx.x * blockDim.x + threadIdx.x;
-    if (cell >= n * n) return;
-    const int row = cell >> k, col = cell & (n - 1);
+    const int pc = blockIdx.x * blockDim.x + threadIdx.x;   // padded cell
+    if (pc >= n * n) return;
+    const int row = pc >> k, col = pc & (n - 1);
     int x = col, y = row;
     int d = 0;
     for (int s = n >> 1; s > 0; s >>= 1) {
@@ -41,56 +45,83 @@ __global__ void hilbert_lut_kernel(int k, int *__restrict__ d2t, int *__restrict
             y = t;
         }
     }
-    t2d[cell] = d;
-    d2t[d] = cell;
-    shared_by_d[d] = (row >= sh_lo && row < sh_hi && col >= sh_lo && col < sh_hi) ? 1 : 0;
+    if (row < H && col < W) {
+        const int cell = row * W + col;
+        pd_of_cell[cell] = d;
+        cell_of_pd[d] = cell;
+        const bool sh = row >= sh_r0 && row < sh_r0 + sh_side && col >= sh_c0 && col < sh_c0 + sh_side;
+        kind_by_pd[d] = sh ? CELL_SHARED : CELL_REAL;
+    } else {
+        cell_of_pd[d] = -1;
+        kind_by_pd[d] = CELL_PAD;
+    }
 }
 
-// c[d] = number of non-shared Hilbert indices below d, for d in [0, HW].
-// Single block; each thread owns a contiguous slice.
-__global__ void nonshared_scan_kernel(const unsigned char *__restrict__ shared_by_d, int HW,
-                                      int *__restrict__ c) {
-    __shared__ int warp_sums[32];
-    __shared__ int carry_sh;
+// c_ns[d] = number of real non-shared cells with padded index below d, c_real[d] =
+// number of real cells below d, for d in [0, NP].  Single block; each thread owns a
+// contiguous slice.
+__global__ void cell_scan_kernel(const unsigned char *__restrict__ kind_by_pd, int NP, int *__restrict__ c_ns,
+                                 int *__restrict__ c_real) {
+    __shared__ int warp_ns[32], warp_real[32];
     const int tid = threadIdx.x;
     const int nthr = blockDim.x;
-    const int per = (HW + nthr - 1) / nthr;
-    const int lo = min(tid * per, HW), hi = min(lo + per, HW);
-    int local = 0;
-    for (int d = lo; d < hi; ++d) local += shared_by_d[d] ? 0 : 1;
-    // block-wide exclusive scan of `local`
-    int v = local;
+    const int per = (NP + nthr - 1) / nthr;
+    const int lo = min(tid * per, NP), hi = min(lo + per, NP);
+    int l_ns = 0, l_real = 0;
+    for (int d = lo; d < hi; ++d) {
+        const unsigned char kd = kind_by_pd[d];
+        l_ns += kd == CELL_REAL;
+        l_real += kd != CELL_PAD;
+    }
+    int v_ns = l_ns, v_real = l_real;
     const int lane = tid & 31, warp = tid >> 5;
     for (int off = 1; off < 32; off <<= 1) {
-        int t = __shfl_up_sync(0xffffffffu, v, off);
-        if (lane >= off) v += t;
+        const int a = __shfl_up_sync(0xffffffffu, v_ns, off), b = __shfl_up_sync(0xffffffffu, v_real, off);
+        if (lane >= off) {
+            v_ns += a;
+            v_real += b;
+        }
     }
-    if (lane == 31) warp_sums[warp] = v;
+    if (lane == 31) {
+        warp_ns[warp] = v_ns;
+        warp_real[warp] = v_real;
+    }
     __syncthreads();
     if (warp == 0) {
-        int w = (lane < (nthr >> 5)) ? warp_sums[lane] : 0;
+        int a = (lane < (nthr >> 5)) ? warp_ns[lane] : 0, b = (lane < (nthr >> 5)) ? warp_real[lane] : 0;
         for (int off = 1; off < 32; off <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, w, off);
-            if (lane >= off) w += t;
+            const int ta = __shfl_up_sync(0xffffffffu, a, off), tb = __shfl_up_sync(0xffffffffu, b, off);
+            if (lane >= off) {
+                a += ta;
+                b += tb;
+            }
         }
-        warp_sums[lane] = w;  // inclusive over warps
+        warp_ns[lane] = a;   // inclusive over warps
+        warp_real[lane] = b;
     }
     __syncthreads();
-    int run = v - local + (warp ? warp_sums[warp - 1] : 0);
+    int run_ns = v_ns - l_ns + (warp ? warp_ns[warp - 1] : 0);
+    int run_real = v_real - l_real + (warp ? warp_real[warp - 1] : 0);
     for (int d = lo; d < hi; ++d) {
-        c[d] = run;
-        run += shared_by_d[d] ? 0 : 1;
+        c_ns[d] = run_ns;
+        c_real[d] = run_real;
+        const unsigned char kd = kind_by_pd[d];
+        run_ns += kd == CELL_REAL;
+        run_real += kd != CELL_PAD;
     }
-    if (tid == nthr - 1) carry_sh = run;
-    __syncthreads();
-    if (tid == 0) c[HW] = carry_sh;
+    if (tid == nthr - 1) {  // the last thread's running totals are the grand totals
+        c_ns[NP] = run_ns;
+        c_real[NP] = run_real;
+    }
 }
 
 // Appendix A layout: text first, then shared tokens, then the rest, each image
-// group by ascending Hilbert index.  One thread per original token.
-__global__ void layout_kernel(int HW, int n_text, int P, int tile, int offset,
-                              const int *__restrict__ t2d, const int *__restrict__ c,
-                              const unsigned char *__restrict__ shared_by_d,
+// group by ascending Hilbert index.  One thread per original token.  Also the
+// rank tables (Hilbert index among the real cells <-> cell).
+__global__ void layout_kernel(int HW, int NP, int n_text, int P, int tile, int offset,
+                              const int *__restrict__ pd_of_cell, const int *__restrict__ c_ns,
+                              const int *__restrict__ c_real, const unsigned char *__restrict__ kind_by_pd,
+                              int *__restrict__ hil_d2t, int *__restrict__ hil_t2d,
                               int *__restrict__ phys2orig, int *__restrict__ orig2phys,
                               int *__restrict__ row_window) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -101,51 +132,49 @@ __global__ void layout_kernel(int HW, int n_text, int P, int tile, int offset,
         row_window[t] = -1;
         return;
     }
-    const int d = t2d[t - n_text];
-    const int below = c[d];
+    const int cell = t - n_text;
+    const int d = pd_of_cell[cell];
+    const int rank = c_real[d];
+    hil_t2d[cell] = rank;
+    hil_d2t[rank] = cell;
+    const int below = c_ns[d];
     int phys;
-    if (shared_by_d[d]) {
-        phys = n_text + (d - below);
+    if (kind_by_pd[d] == CELL_SHARED) {
+        phys = n_text + (rank - below);
         row_window[phys] = -1;
     } else {
         phys = P + below;
-        row_window[phys] = ((d + offset) % HW) / tile;
+        row_window[phys] = ((d + offset) % NP) / tile;
     }
     phys2orig[phys] = t;
     orig2phys[t] = phys;
 }
 
-// Sec. 3.2 with wrap-around: slid tile w covers Hilbert indices
-// [w*tile - offset, +tile) mod HW; its non-shared members are contiguous in the
-// physical order, in one range or two if the interval wraps.
-__global__ void window_kernel(int HW, int T, int tile, int offset, int P, const int *__restrict__ c,
+// Sec. 3.2 with wrap-around: slid tile w covers (padded) Hilbert indices
+// [w*tile - offset, +tile) mod NP; its real non-shared members are contiguous in
+// the physical order, in one range or two if the interval wraps.
+__global__ void window_kernel(int NP, int T, int tile, int offset, int P, const int *__restrict__ c,
                               Window *__restrict__ win) {
     const int w = blockIdx.x * blockDim.x + threadIdx.x;
     if (w >= T) return;
-    long long lo_ll = ((long long)w * tile - offset) % HW;
-    if (lo_ll < 0) lo_ll += HW;
+    long long lo_ll = ((long long)w * tile - offset) % NP;
+    if (lo_ll < 0) lo_ll += NP;
     const int lo = (int)lo_ll;
     const int hi = lo + tile;
     Window r;
     r.lo = lo;
-    const int a0 = lo, b0 = hi <= HW ? hi : HW;
+    const int a0 = lo, b0 = hi <= NP ? hi : NP;
     const int n0 = c[b0] - c[a0];
     r.seg0_start = n0 > 0 ? P + c[a0] : 0;
     r.seg0_len = n0;
     r.seg1_start = 0;
     r.seg1_len = 0;
-    if (hi > HW) {
-        const int n1 = c[hi - HW] - c[0];
+    if (hi > NP) {
+        const int n1 = c[hi - NP] - c[0];
         r.seg1_start = n1 > 0 ? P + c[0] : 0;
         r.seg1_len = n1;
     }
     win[w] = r;
-}
-
-static int ilog2_exact(int n) {
-    int k = 0;
-    while ((1 << k) < n) ++k;
-    return ((1 << k) == n) ? k : -1;
 }
 
 static void free_plan(hilberta_plan_t *p) {
@@ -166,36 +195,44 @@ static void free_plan(hilberta_plan_t *p) {
 }
 
 static int build_plan(hilberta_plan_t *p) {
-    const int HW = p->HW, S = p->S;
-    unsigned char *d_shared = nullptr;
+    const int HW = p->HW, S = p->S, NP = p->NP;
+    unsigned char *d_kind = nullptr;
+    int *d_cell_of_pd = nullptr, *d_pd_of_cell = nullptr, *d_c_real = nullptr;
     HB_CUDA(cudaMalloc(&p->d_hil_d2t, sizeof(int) * HW));
     HB_CUDA(cudaMalloc(&p->d_hil_t2d, sizeof(int) * HW));
-    HB_CUDA(cudaMalloc(&p->d_c, sizeof(int) * (HW + 1)));
+    HB_CUDA(cudaMalloc(&p->d_c, sizeof(int) * (NP + 1)));
     HB_CUDA(cudaMalloc(&p->d_phys2orig, sizeof(int) * S));
     HB_CUDA(cudaMalloc(&p->d_orig2phys, sizeof(int) * S));
     HB_CUDA(cudaMalloc(&p->d_row_window, sizeof(int) * S));
     HB_CUDA(cudaMalloc(&p->d_windows, sizeof(Window) * p->T));
     HB_CUDA(cudaMalloc(&p->d_status, sizeof(int) * 4096));
     HB_CUDA(cudaMemset(p->d_status, 0, sizeof(int) * 4096));
-    HB_CUDA(cudaMalloc(&d_shared, HW));
 
-    const int sh_lo = p->H / 2 - p->shared_region / 2;
-    const int sh_hi = sh_lo + p->shared_region;
+    const int sh_r0 = p->H / 2 - p->shared_region / 2;
+    const int sh_c0 = p->W / 2 - p->shared_region / 2;
     int rc = HILBERTA_OK;
     do {
-        hilbert_lut_kernel<<<(HW + 255) / 256, 256>>>(p->k_log2, p->d_hil_d2t, p->d_hil_t2d, d_shared,
-                                                      sh_lo, sh_hi);
+        cudaError_t e = cudaMalloc(&d_kind, NP);
+        if (e == cudaSuccess) e = cudaMalloc(&d_cell_of_pd, sizeof(int) * NP);
+        if (e == cudaSuccess) e = cudaMalloc(&d_pd_of_cell, sizeof(int) * HW);
+        if (e == cudaSuccess) e = cudaMalloc(&d_c_real, sizeof(int) * (NP + 1));
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            rc = HILBERTA_ERR_CUDA;
+            break;
+        }
+        hilbert_lut_kernel<<<(NP + 255) / 256, 256>>>(p->k_log2, p->H, p->W, d_cell_of_pd, d_pd_of_cell, d_kind,
+                                                      sh_r0, sh_c0, p->shared_region);
         g_launches.fetch_add(1);
-        nonshared_scan_kernel<<<1, 1024>>>(d_shared, HW, p->d_c);
+        cell_scan_kernel<<<1, 1024>>>(d_kind, NP, p->d_c, d_c_real);
         g_launches.fetch_add(1);
-        layout_kernel<<<(S + 255) / 256, 256>>>(HW, p->n_text, p->P, p->tile, p->offset, p->d_hil_t2d,
-                                                p->d_c, d_shared, p->d_phys2orig, p->d_orig2phys,
-                                                p->d_row_window);
+        layout_kernel<<<(S + 255) / 256, 256>>>(HW, NP, p->n_text, p->P, p->tile, p->offset, d_pd_of_cell, p->d_c,
+                                                d_c_real, d_kind, p->d_hil_d2t, p->d_hil_t2d, p->d_phys2orig,
+                                                p->d_orig2phys, p->d_row_window);
         g_launches.fetch_add(1);
-        window_kernel<<<(p->T + 127) / 128, 128>>>(HW, p->T, p->tile, p->offset, p->P, p->d_c,
-                                                   p->d_windows);
+        window_kernel<<<(p->T + 127) / 128, 128>>>(NP, p->T, p->tile, p->offset, p->P, p->d_c, p->d_windows);
         g_launches.fetch_add(1);
-        cudaError_t e = cudaGetLastError();
+        e = cudaGetLastError();
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
         if (e != cudaSuccess) {
             g_last_cuda_error = (int)e;
@@ -204,17 +241,17 @@ static int build_plan(hilberta_plan_t *p) {
         }
         // host mirrors of the small tables
         p->h_windows.resize(p->T);
-        std::vector<unsigned char> h_shared(HW);
+        std::vector<unsigned char> h_kind(NP);
         e = cudaMemcpy(p->h_windows.data(), p->d_windows, sizeof(Window) * p->T, cudaMemcpyDeviceToHost);
-        if (e == cudaSuccess) e = cudaMemcpy(h_shared.data(), d_shared, HW, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) e = cudaMemcpy(h_kind.data(), d_kind, NP, cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) {
             g_last_cuda_error = (int)e;
             rc = HILBERTA_ERR_CUDA;
             break;
         }
         int n_sh = 0;
-        for (int d = 0; d < HW; ++d) {
-            if (!h_shared[d]) continue;
+        for (int d = 0; d < NP; ++d) {
+            if (h_kind[d] != CELL_SHARED) continue;
             ++n_sh;
             size_t n = p->h_shared_runs.size();
             if (n && p->h_shared_runs[n - 2] + p->h_shared_runs[n - 1] == d) {
@@ -238,7 +275,10 @@ static int build_plan(hilberta_plan_t *p) {
         }
         p->nnz = nnz;
     } while (0);
-    cudaFree(d_shared);
+    cudaFree(d_kind);
+    cudaFree(d_cell_of_pd);
+    cudaFree(d_pd_of_cell);
+    cudaFree(d_c_real);
     return rc;
 }
 
@@ -251,10 +291,13 @@ extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int share
     if (!out) return HILBERTA_ERR_INVALID;
     *out = nullptr;
     if (H < 1 || W < 1 || n_text < 0 || tile < 1 || shared_region < 0) return HILBERTA_ERR_INVALID;
-    if (H != W || ilog2_exact(H) < 0 || H > 1024) return HILBERTA_ERR_UNSUPPORTED;
+    if (H > 1024 || W > 1024) return HILBERTA_ERR_UNSUPPORTED;
     const int HW = H * W;
-    if (HW % tile) return HILBERTA_ERR_INVALID;
-    if (shared_region % 2 || shared_region > H) return HILBERTA_ERR_INVALID;
+    int k_log2 = 0;                       // padded side n = 2^k >= max(H, W)
+    while ((1 << k_log2) < (H > W ? H : W)) ++k_log2;
+    const int NP = 1 << (2 * k_log2);     // length of the padded curve
+    if (NP % tile) return HILBERTA_ERR_INVALID;
+    if (shared_region % 2 || shared_region > H || shared_region > W) return HILBERTA_ERR_INVALID;
     if ((long long)n_text + HW > (1ll << 30)) return HILBERTA_ERR_INVALID;
 
     int dev = 0;
@@ -270,15 +313,16 @@ extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int share
     p->H = H;
     p->W = W;
     p->HW = HW;
-    p->k_log2 = ilog2_exact(H);
+    p->NP = NP;
+    p->k_log2 = k_log2;
     p->tile = tile;
-    long long o = (long long)layer_offset % HW;
-    if (o < 0) o += HW;
+    long long o = (long long)layer_offset % NP;
+    if (o < 0) o += NP;
     p->offset = (int)o;
     p->shared_region = shared_region;
     p->n_text = n_text;
     p->n_shared = shared_region * shared_region;
-    p->T = HW / tile;
+    p->T = NP / tile;
     p->S = n_text + HW;
     p->P = n_text + p->n_shared;
     p->bound = false;
@@ -319,7 +363,7 @@ extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *ho
             break;
         case HILBERTA_EXPORT_NNZ: need = sizeof(uint64_t); hsrc = &nnz; break;
         case HILBERTA_EXPORT_INFO:
-            tmp = {p->H, p->W, p->tile, p->offset, p->shared_region, p->n_text, p->n_shared, p->T};
+            tmp = {p->H, p->W, p->tile, p->offset, p->shared_region, p->n_text, p->n_shared, p->T, 1 << p->k_log2};
             need = sizeof(int) * tmp.size();
             hsrc = tmp.data();
             break;

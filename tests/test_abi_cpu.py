@@ -47,8 +47,9 @@ def test_argument_validation_needs_no_device(lib):
     ]
     for args in bad:
         assert lib.hilberta_plan(*args, ctypes.byref(h)) == binding.ERR_INVALID
-    assert lib.hilberta_plan(8, 16, 16, 0, 0, 0, ctypes.byref(h)) == binding.ERR_UNSUPPORTED
-    assert lib.hilberta_plan(12, 12, 16, 0, 0, 0, ctypes.byref(h)) == binding.ERR_UNSUPPORTED
+    assert lib.hilberta_plan(2048, 16, 16, 0, 0, 0, ctypes.byref(h)) == binding.ERR_UNSUPPORTED
+    assert lib.hilberta_plan(12, 12, 48, 0, 0, 0, ctypes.byref(h)) == binding.ERR_INVALID  # 48 does not divide 16*16
+    assert lib.hilberta_plan(8, 16, 16, 0, 10, 0, ctypes.byref(h)) == binding.ERR_INVALID  # shared side > H
     assert lib.hilberta_plan(8, 8, 5, 0, 0, 0, ctypes.byref(h)) == binding.ERR_INVALID
     assert lib.hilberta_plan(8, 8, 16, 0, 3, 0, ctypes.byref(h)) == binding.ERR_INVALID
     assert lib.hilberta_plan(8, 8, 16, 0, 10, 0, ctypes.byref(h)) == binding.ERR_INVALID

@@ -185,3 +185,19 @@ def test_forward_unpermute_equals_forward_then_unpermute():
             assert torch.equal(out_a.view(view), out_b.view(view))
         finally:
             plan.destroy()
+
+
+@pytest.mark.parametrize("H,W,tile,o,hs,nt", [(24, 40, 256, 100, 4, 77), (48, 32, 512, 256, 8, 130), (5, 3, 16, 3, 2, 40)])
+def test_general_shapes_elementwise(H, W, tile, o, hs, nt):
+    """Non-square / non-power-of-two grids: same kernels, plan built on the padded curve."""
+    S = nt + H * W
+    g = torch.Generator().manual_seed(4242 + H)
+    q, k, v = (torch.randn((1, 2, S, 128), generator=g).bfloat16() for _ in range(3))
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    try:
+        got = run_gpu(plan, q, k, v)
+    finally:
+        plan.destroy()
+    ig, grp = orc.token_classes(H, W, tile, o, hs, nt)
+    ref = attn_c.attention_rows(q.float().numpy(), k.float().numpy(), v.float().numpy(), ig, grp)
+    check(got, ref)

@@ -126,3 +126,18 @@ def test_forward_errors():
         assert L.hilberta_forward(x.data_ptr(), x.data_ptr(), x.data_ptr(), None, plan._h, None) == hb.ERR_INVALID
     finally:
         plan.destroy()
+
+
+def test_general_shape_fp32():
+    H, W, tile, o, hs, nt = 12, 20, 64, 19, 4, 7
+    S = nt + H * W
+    g = torch.Generator().manual_seed(8)
+    q, k, v = (torch.randn((1, 2, S, 64), generator=g) for _ in range(3))
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    try:
+        got = run_gpu(plan, q, k, v).double().numpy()
+    finally:
+        plan.destroy()
+    ig, grp = orc.token_classes(H, W, tile, o, hs, nt)
+    ref = attn_c.attention_rows(q.numpy(), k.numpy(), v.numpy(), ig, grp)
+    assert orc.max_abs_err(got, ref) <= TOL_FP32 and orc.rel_l2_err(got, ref) <= TOL_FP32

@@ -9,9 +9,10 @@ from paper_2509_26538_b200.inputs import TINY_LAYER_OFFSETS, WORKLOADS
 pytestmark = pytest.mark.gpu
 
 
-def _check(H, tile, o, hs, nt):
-    ref = orc.plan_arrays(H, H, tile, o, hs, nt)
-    plan = hb.Plan(H, H, tile, o, hs, nt)
+def _check(H, tile, o, hs, nt, W=None):
+    W = H if W is None else W
+    ref = orc.plan_arrays(H, W, tile, o, hs, nt)
+    plan = hb.Plan(H, W, tile, o, hs, nt)
     try:
         assert np.array_equal(plan.export(hb.EXPORT_HIL_D2T), ref["hil_d2t"])
         assert np.array_equal(plan.export(hb.EXPORT_HIL_T2D), ref["hil_t2d"])
@@ -21,8 +22,8 @@ def _check(H, tile, o, hs, nt):
         assert np.array_equal(plan.export(hb.EXPORT_WINDOWS), ref["windows"])
         assert int(plan.export(hb.EXPORT_NNZ)[0]) == ref["nnz"]
         info = plan.export(hb.EXPORT_INFO).tolist()
-        HW = H * H
-        assert info == [H, H, tile, o % HW, hs, nt, hs * hs, HW // tile]
+        NP = orc.padded_side(H, W) ** 2
+        assert info == [H, W, tile, o % NP, hs, nt, hs * hs, NP // tile, orc.padded_side(H, W)]
     finally:
         plan.destroy()
 
@@ -77,6 +78,22 @@ def test_random_small_geometries():
             assert int(plan.export(hb.EXPORT_NNZ)[0]) == ref["nnz"]
         finally:
             plan.destroy()
+
+
+def test_general_shapes():
+    """Non-square and non-power-of-two grids (appendix on general shapes)."""
+    _check(24, 256, 100, 4, 77, W=40)      # padded to 64 x 64
+    _check(3, 8, 3, 2, 2, W=5)
+    _check(96, 1024, 512, 8, 512, W=128)   # a 3:4 latent grid
+    _check(1, 16, 7, 0, 1, W=9)
+    _check(100, 4096, 1024, 16, 0, W=100)
+    rng = np.random.default_rng(11)
+    for _ in range(25):
+        H, W = int(rng.integers(1, 40)), int(rng.integers(1, 40))
+        NP = orc.padded_side(H, W) ** 2
+        tile = int(rng.choice([t for t in (1, 2, 4, 8, 16, 32, 64, 128, 256, 1024, 4096) if NP % t == 0]))
+        hs = int(rng.choice([s for s in range(0, min(H, W) + 1, 2)]))
+        _check(H, tile, int(rng.integers(-NP, 2 * NP)), hs, int(rng.choice([0, 3, 50])), W=W)
 
 
 def test_degenerate_and_maximum():
