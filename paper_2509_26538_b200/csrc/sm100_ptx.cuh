@@ -45,19 +45,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// try_wait that lets the hardware park the thread for up to `ns` nanoseconds (it
-// still resumes as soon as the phase completes): for roles that wait a long time.
-__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, P;\n\t}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(ns)
-        : "memory");
-    return ok != 0;
-}
 // Bounded wait: returns false (and the caller bails out) if the phase never
 // completes.  Each try_wait already blocks for a hardware-defined slice.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_tries = (1u << 22)) {
@@ -152,7 +139,6 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 }
 
 // ---- TMEM <-> registers: 32 lanes x 32-bit, N consecutive columns per thread.
-#define HB_R4(a, i) "%" #a
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -185,7 +171,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
           "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr)
         : "memory");
 }
-#undef HB_R4
 
 }  // namespace ptx
 }  // namespace hilberta
