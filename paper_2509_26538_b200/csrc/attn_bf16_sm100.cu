@@ -699,42 +699,3 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
 }
 
 }  // namespace hilberta
-
-// Whole path for host-resident activations: H2D copies, three entry gathers,
-// forward, exit gather, D2H copy.  Seven device buffers of one tensor each.
-extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v, void *out,
-                                     hilberta_plan_t *p, void *stream) {
-    if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
-    if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    const int64_t dense_h = (int64_t)p->S * p->head_dim;
-    if (p->stride_s != p->head_dim || p->stride_h != dense_h || p->stride_b != dense_h * p->heads)
-        return HILBERTA_ERR_INVALID;
-    const size_t esz = p->dtype == HILBERTA_BF16 ? 2 : 4;
-    const size_t bytes = (size_t)p->batch * p->heads * p->S * p->head_dim * esz;
-    const size_t slot = (bytes + 255) & ~(size_t)255;
-    if (p->ws_bytes < 7 * slot) {
-        cudaFree(p->ws);
-        p->ws = nullptr;
-        p->ws_bytes = 0;
-        HB_CUDA(cudaMalloc(&p->ws, 7 * slot));
-        p->ws_bytes = 7 * slot;
-    }
-    cudaStream_t st = (cudaStream_t)stream;
-    char *ws = (char *)p->ws;
-    void *in[3] = {ws, ws + slot, ws + 2 * slot};
-    void *perm[3] = {ws + 3 * slot, ws + 4 * slot, ws + 5 * slot};
-    void *out_phys = ws + 6 * slot;
-    const void *host_in[3] = {q, k, v};
-    const int bh = p->batch * p->heads;
-    for (int i = 0; i < 3; ++i) {
-        HB_CUDA(cudaMemcpyAsync(in[i], host_in[i], bytes, cudaMemcpyHostToDevice, st));
-        int rc = hilberta_permute(in[i], perm[i], p, bh, p->head_dim, p->dtype, st);
-        if (rc != HILBERTA_OK) return rc;
-    }
-    (void)bh;
-    int rc = hilberta_forward_unpermute(perm[0], perm[1], perm[2], out_phys, p, st);  // out_phys holds ORIGINAL order
-    if (rc != HILBERTA_OK) return rc;
-    HB_CUDA(cudaMemcpyAsync(out, out_phys, bytes, cudaMemcpyDeviceToHost, st));
-    HB_CUDA(cudaStreamSynchronize(st));
-    return HILBERTA_OK;
-}
