@@ -27,6 +27,8 @@ Where each piece comes from
   text tokens are treated exactly like the shared anchor region).
 * attention : softmax(s * q k^T restricted to the mask) v, the quantity
   Algorithm 1's online softmax reaches up to rounding.
+* token_classes_compact / mask_compact / plan_arrays_compact : Appendix A read
+  literally (Algorithm 1's S = N / G over the non-shared tokens).
 * plan arrays : the memory layout of Appendix A (prefix of text + shared
   tokens, then the remaining image tokens in Hilbert order) and the contiguous
   key ranges of each slid tile ("pointer shift", modular indexing, Sec. 3.2/3.4).
@@ -337,6 +339,80 @@ def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
         "prefix": int(P),
         "padded_side": int(n),
     }
+
+
+# --------------------------------------------------------------------------
+# Appendix A read literally: G equal groups over the NON-SHARED tokens
+# --------------------------------------------------------------------------
+
+
+def token_classes_compact(H, W, groups, layer_offset, shared_region, n_text):
+    """Per original token: is_global and group, for the group arithmetic of Algorithm 1.
+
+    There the shared tokens are taken out first; the remaining R = HW - n_shared image
+    tokens, in Hilbert order, form a sequence of their own that is cut into `groups`
+    equal groups of R / groups tokens (S = N / G, start = group_id * S).  The slide of
+    Sec. 3.2 is applied to positions in that sequence.  With no shared region this is
+    the same mask as token_classes(tile = HW / groups)."""
+    HW = H * W
+    S = n_text + HW
+    pidx = hilbert_cell_index(H, W)
+    is_global = np.zeros(S, dtype=np.uint8)
+    is_global[:n_text] = 1
+    sh_cells = shared_cells(H, W, shared_region)
+    is_global[n_text + sh_cells] = 1
+    R = HW - sh_cells.size
+    if groups < 1 or R % groups:
+        raise ValueError("groups must divide the number of non-shared image tokens")
+    size = R // groups if R else 1
+    group = np.full(S, -1, dtype=np.int32)
+    order = np.argsort(pidx, kind="stable")               # cells in curve order
+    nonshared = [c for c in order.tolist() if not is_global[n_text + c]]
+    for pos, c in enumerate(nonshared):
+        group[n_text + c] = ((pos + int(layer_offset)) % R) // size
+    # shared image tokens are global; give them a tile id that matches nobody else
+    for c in sh_cells.tolist():
+        group[n_text + c] = groups
+    return is_global, group
+
+
+def mask_compact(H, W, groups, layer_offset, shared_region, n_text) -> np.ndarray:
+    is_global, group = token_classes_compact(H, W, groups, layer_offset, shared_region, n_text)
+    g = is_global.astype(bool)
+    img = (group >= 0) & ~g
+    same = (group[:, None] == group[None, :]) & img[:, None] & img[None, :]
+    return g[:, None] | g[None, :] | same
+
+
+def plan_arrays_compact(H, W, groups, layer_offset, shared_region, n_text) -> dict:
+    """Canonical arrays for the compact tiling: same physical order as plan_arrays;
+    windows[w] = (lo, seg0_start, seg0_len, seg1_start, seg1_len) with lo the position in
+    the non-shared sequence where group w starts."""
+    base = plan_arrays(H, W, padded_side(H, W) ** 2, 0, shared_region, n_text)   # layout only
+    HW = H * W
+    S = n_text + HW
+    P = base["prefix"]
+    R = S - P
+    if groups < 1 or R % groups:
+        raise ValueError("groups must divide the number of non-shared image tokens")
+    size = R // groups if R else 0
+    o = int(layer_offset) % R if R else 0
+    windows = np.zeros((groups, 5), dtype=np.int32)
+    for w in range(groups):
+        if size == 0:
+            continue
+        lo = (w * size - o) % R
+        hi = lo + size
+        if hi <= R:
+            windows[w] = [lo, P + lo, size, 0, 0]
+        else:
+            windows[w] = [lo, P + lo, R - lo, P, hi - R]
+    is_global, group = token_classes_compact(H, W, groups, layer_offset, shared_region, n_text)
+    n_glob = int(is_global.sum())
+    total = n_glob * S + groups * size * (n_glob + size)
+    out = dict(base)
+    out.update({"windows": windows, "nnz": int(total)})
+    return out
 
 
 def permute_rows(x, phys2orig):

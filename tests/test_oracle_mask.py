@@ -253,3 +253,64 @@ def test_permute_roundtrip():
     y = orc.permute_rows(x, p["phys2orig"])
     assert np.array_equal(y[:, 7], x[:, p["phys2orig"][7]])
     assert np.array_equal(orc.unpermute_rows(y, p["phys2orig"]), x)
+
+
+# ---- Appendix A group arithmetic (equal groups over the non-shared tokens) ----
+
+def _naive_mask_compact(H, W, groups, o, hs, n_text):
+    n = 1
+    while n < max(H, W):
+        n *= 2
+    pts = orc.hilbert_points(int(np.log2(n)))
+    r0, c0 = H // 2 - hs // 2, W // 2 - hs // 2
+    shared = lambda r, c: r0 <= r < r0 + hs and c0 <= c < c0 + hs
+    seq = [(y, x) for (x, y) in pts if y < H and x < W and not shared(y, x)]   # non-shared cells in curve order
+    R = len(seq)
+    size = R // groups
+    gid = {cell: ((pos + o) % R) // size for pos, cell in enumerate(seq)}
+    S = n_text + H * W
+    M = np.zeros((S, S), dtype=bool)
+    for i in range(S):
+        for j in range(S):
+            gi = i < n_text or (divmod(i - n_text, W) not in gid)
+            gj = j < n_text or (divmod(j - n_text, W) not in gid)
+            M[i, j] = gi or gj or gid[divmod(i - n_text, W)] == gid[divmod(j - n_text, W)]
+    return M
+
+
+@pytest.mark.parametrize("H,W,groups,o,hs,n_text", [
+    (8, 8, 4, 0, 2, 3), (8, 8, 5, 7, 2, 0), (8, 8, 12, 100, 2, 1), (4, 4, 3, 2, 2, 2), (6, 4, 4, 3, 2, 1),
+    (8, 8, 4, 9, 0, 2),
+])
+def test_compact_tiling_bruteforce(H, W, groups, o, hs, n_text):
+    M = orc.mask_compact(H, W, groups, o, hs, n_text)
+    assert np.array_equal(M, _naive_mask_compact(H, W, groups, o, hs, n_text))
+    assert np.array_equal(M, M.T) and M.diagonal().all()
+    p = orc.plan_arrays_compact(H, W, groups, o, hs, n_text)
+    assert p["nnz"] == int(M.sum())
+    S, P, p2o = M.shape[0], p["prefix"], p["phys2orig"]
+    Mp = np.zeros((S, S), dtype=bool)
+    Mp[:P, :] = True
+    Mp[:, :P] = True
+    covered = np.zeros(S, dtype=int)
+    for (lo, s0, n0, s1, n1) in p["windows"].tolist():
+        idx = list(range(s0, s0 + n0)) + list(range(s1, s1 + n1))
+        covered[idx] += 1
+        Mp[np.ix_(idx, idx)] = True
+    assert np.all(covered[P:] == 1)
+    assert np.array_equal(Mp, M[np.ix_(p2o, p2o)])
+
+
+def test_compact_equals_curve_tiling_without_shared_region():
+    for (H, groups, o, nt) in [(8, 4, 5, 3), (16, 8, 40, 0)]:
+        A = orc.mask(H, H, H * H // groups, o, 0, nt)
+        B = orc.mask_compact(H, H, groups, o, 0, nt)
+        assert np.array_equal(A, B)
+
+
+def test_compact_matches_table1_group_sizes():
+    """Table 1's settings: 16x16 shared at 1024^2 leaves 3840 tokens -> 960 / 240 per group."""
+    p = orc.plan_arrays_compact(64, 64, 4, 0, 16, 512)
+    assert p["windows"][:, 2].tolist() == [960] * 4 and p["prefix"] == 768
+    p = orc.plan_arrays_compact(64, 64, 16, 60, 16, 512)
+    assert (p["windows"][:, 2] + p["windows"][:, 4]).tolist() == [240] * 16
