@@ -195,6 +195,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="flux2048")
     ap.add_argument("--tile", type=int, default=0)
+    ap.add_argument("--groups", type=int, default=0,
+                    help="use the Appendix-A tiling with this many equal groups over the non-shared tokens "
+                         "(the paper's Table 1 settings: --groups 4|16 --shared 16 at 1024^2, 32 at 2048^2)")
+    ap.add_argument("--shared", type=int, default=-1, help="override the side of the central shared region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--schedule", action="store_true",
@@ -207,6 +211,13 @@ def main():
     wl = WORKLOADS[args.workload]
     if args.tile:
         wl = wl.with_(tile=args.tile, layer_offset=args.tile // 2)
+    if args.shared >= 0:
+        wl = wl.with_(shared_region=args.shared)
+    if args.groups:
+        if args.impl == "reference" or args.schedule:
+            raise SystemExit("--groups is a timing-only option of the CUDA arm")
+        size = (wl.HW - wl.shared_region ** 2) // args.groups
+        wl = wl.with_(tile=size, layer_offset=size // 2, name=wl.name + f"-groups{args.groups}")
 
     if args.impl == "reference":
         run_reference(args, wl)
@@ -237,7 +248,7 @@ def main():
     qp, kp, vp, op, od = (torch.empty_like(qd) for _ in range(5))
 
     t0 = time.perf_counter()
-    plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
+    plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text, groups=args.groups)
     plan.bind_like(qp)
     torch.cuda.synchronize()
     plan_ms = 1e3 * (time.perf_counter() - t0)
@@ -399,7 +410,7 @@ def main():
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
                              "(4.36 ms per call at 2048^2, 16 tiles)"},
     }
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and not args.groups:
         tf, threads, desc, dt = oracle_sample(wl, 15.0)
         line["cpu_baseline"] = {"value": tf, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
                                 "sample": desc, "seconds": dt}

@@ -97,6 +97,19 @@ typedef struct hilberta_plan_s hilberta_plan_t;
 int hilberta_plan(int H, int W, int tile, int layer_offset, int shared_region, int n_text,
                   hilberta_plan_t **out);
 
+/* The same plan with the tiles of Appendix A / Algorithm 1 read literally (S = N / G,
+ * start = group_id * S): the shared tokens are taken out first, and the remaining
+ * R = H*W - shared_region^2 image tokens, in curve order, are cut into `groups` equal
+ * groups of R / groups tokens; `layer_offset` slides the group boundaries along that
+ * sequence (reduced modulo R).  groups >= 1 and R % groups == 0, else ERR_INVALID.
+ * With shared_region = 0 on a power-of-two square this is hilberta_plan with
+ * tile = H*W / groups.  The exported window table has `groups` rows whose `lo` is the
+ * position in the non-shared sequence.  Everything downstream (bind, forward, permute)
+ * is the same.  This is the tiling the paper's Table 1 settings use (16 x 16 shared
+ * region at 1024^2: groups of 960 or 240 tokens). */
+int hilberta_plan_groups(int H, int W, int groups, int layer_offset, int shared_region, int n_text,
+                         hilberta_plan_t **out);
+
 /* Free a plan and every device table it owns.  NULL is accepted. */
 int hilberta_plan_destroy(hilberta_plan_t *plan);
 

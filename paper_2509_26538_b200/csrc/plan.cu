@@ -118,7 +118,9 @@ __global__ void cell_scan_kernel(const unsigned char *__restrict__ kind_by_pd, i
 // Appendix A layout: text first, then shared tokens, then the rest, each image
 // group by ascending Hilbert index.  One thread per original token.  Also the
 // rank tables (Hilbert index among the real cells <-> cell).
-__global__ void layout_kernel(int HW, int NP, int n_text, int P, int tile, int offset,
+// compact_R > 0 selects the group arithmetic of Algorithm 1: tile ids follow the position
+// in the non-shared sequence (c_ns) instead of the position on the padded curve.
+__global__ void layout_kernel(int HW, int NP, int n_text, int P, int tile, int offset, int compact_R,
                               const int *__restrict__ pd_of_cell, const int *__restrict__ c_ns,
                               const int *__restrict__ c_real, const unsigned char *__restrict__ kind_by_pd,
                               int *__restrict__ hil_d2t, int *__restrict__ hil_t2d,
@@ -144,7 +146,7 @@ __global__ void layout_kernel(int HW, int NP, int n_text, int P, int tile, int o
         row_window[phys] = -1;
     } else {
         phys = P + below;
-        row_window[phys] = ((d + offset) % NP) / tile;
+        row_window[phys] = compact_R > 0 ? ((below + offset) % compact_R) / tile : ((d + offset) % NP) / tile;
     }
     phys2orig[phys] = t;
     orig2phys[t] = phys;
@@ -174,6 +176,23 @@ __global__ void window_kernel(int NP, int T, int tile, int offset, int P, const 
         r.seg1_start = n1 > 0 ? P + c[0] : 0;
         r.seg1_len = n1;
     }
+    win[w] = r;
+}
+
+// Appendix A / Algorithm 1 read literally: `groups` equal groups of `size` tokens over
+// the R non-shared tokens in curve order, slid by `offset` positions of that sequence.
+__global__ void window_compact_kernel(int R, int groups, int size, int offset, int P, Window *__restrict__ win) {
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w >= groups) return;
+    Window r;
+    long long lo_ll = ((long long)w * size - offset) % R;
+    if (lo_ll < 0) lo_ll += R;
+    const int lo = (int)lo_ll;
+    r.lo = lo;
+    r.seg0_start = P + lo;
+    r.seg0_len = lo + size <= R ? size : R - lo;
+    r.seg1_start = lo + size <= R ? 0 : P;
+    r.seg1_len = lo + size <= R ? 0 : lo + size - R;
     win[w] = r;
 }
 
@@ -226,11 +245,15 @@ static int build_plan(hilberta_plan_t *p) {
         g_launches.fetch_add(1);
         cell_scan_kernel<<<1, 1024>>>(d_kind, NP, p->d_c, d_c_real);
         g_launches.fetch_add(1);
-        layout_kernel<<<(S + 255) / 256, 256>>>(HW, NP, p->n_text, p->P, p->tile, p->offset, d_pd_of_cell, p->d_c,
+        layout_kernel<<<(S + 255) / 256, 256>>>(HW, NP, p->n_text, p->P, p->tile, p->offset,
+                                                p->compact ? S - p->P : 0, d_pd_of_cell, p->d_c,
                                                 d_c_real, d_kind, p->d_hil_d2t, p->d_hil_t2d, p->d_phys2orig,
                                                 p->d_orig2phys, p->d_row_window);
         g_launches.fetch_add(1);
-        window_kernel<<<(p->T + 127) / 128, 128>>>(NP, p->T, p->tile, p->offset, p->P, p->d_c, p->d_windows);
+        if (p->compact)
+            window_compact_kernel<<<(p->T + 127) / 128, 128>>>(S - p->P, p->T, p->tile, p->offset, p->P, p->d_windows);
+        else
+            window_kernel<<<(p->T + 127) / 128, 128>>>(NP, p->T, p->tile, p->offset, p->P, p->d_c, p->d_windows);
         g_launches.fetch_add(1);
         e = cudaGetLastError();
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -286,19 +309,29 @@ static int build_plan(hilberta_plan_t *p) {
 
 using namespace hilberta;
 
-extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int shared_region, int n_text,
-                             hilberta_plan_t **out) {
+// tile > 0: curve tiling (tiles of `tile` positions of the padded curve).
+// groups > 0: compact tiling (Algorithm 1's equal groups over the non-shared tokens).
+static int make_plan(int H, int W, int tile, int groups, int layer_offset, int shared_region, int n_text,
+                     hilberta_plan_t **out) {
     if (!out) return HILBERTA_ERR_INVALID;
     *out = nullptr;
-    if (H < 1 || W < 1 || n_text < 0 || tile < 1 || shared_region < 0) return HILBERTA_ERR_INVALID;
+    const bool compact = groups > 0;
+    if (H < 1 || W < 1 || n_text < 0 || shared_region < 0) return HILBERTA_ERR_INVALID;
+    if (!compact && tile < 1) return HILBERTA_ERR_INVALID;
     if (H > 1024 || W > 1024) return HILBERTA_ERR_UNSUPPORTED;
     const int HW = H * W;
     int k_log2 = 0;                       // padded side n = 2^k >= max(H, W)
     while ((1 << k_log2) < (H > W ? H : W)) ++k_log2;
     const int NP = 1 << (2 * k_log2);     // length of the padded curve
-    if (NP % tile) return HILBERTA_ERR_INVALID;
     if (shared_region % 2 || shared_region > H || shared_region > W) return HILBERTA_ERR_INVALID;
     if ((long long)n_text + HW > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    const int R = HW - shared_region * shared_region;   // non-shared image tokens
+    if (compact) {
+        if (R < 1 || R % groups) return HILBERTA_ERR_INVALID;
+        tile = R / groups;
+    } else if (NP % tile) {
+        return HILBERTA_ERR_INVALID;
+    }
 
     int dev = 0;
     HB_CUDA(cudaGetDevice(&dev));
@@ -315,14 +348,16 @@ extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int share
     p->HW = HW;
     p->NP = NP;
     p->k_log2 = k_log2;
+    p->compact = compact;
     p->tile = tile;
-    long long o = (long long)layer_offset % NP;
-    if (o < 0) o += NP;
+    const long long period = compact ? R : NP;
+    long long o = (long long)layer_offset % period;
+    if (o < 0) o += period;
     p->offset = (int)o;
     p->shared_region = shared_region;
     p->n_text = n_text;
     p->n_shared = shared_region * shared_region;
-    p->T = NP / tile;
+    p->T = compact ? groups : NP / tile;
     p->S = n_text + HW;
     p->P = n_text + p->n_shared;
     p->bound = false;
@@ -333,6 +368,24 @@ extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int share
     }
     *out = p;
     return HILBERTA_OK;
+}
+
+extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int shared_region, int n_text,
+                             hilberta_plan_t **out) {
+    if (tile < 1) {
+        if (out) *out = nullptr;
+        return HILBERTA_ERR_INVALID;
+    }
+    return make_plan(H, W, tile, 0, layer_offset, shared_region, n_text, out);
+}
+
+extern "C" int hilberta_plan_groups(int H, int W, int groups, int layer_offset, int shared_region, int n_text,
+                                    hilberta_plan_t **out) {
+    if (groups < 1) {
+        if (out) *out = nullptr;
+        return HILBERTA_ERR_INVALID;
+    }
+    return make_plan(H, W, 0, groups, layer_offset, shared_region, n_text, out);
 }
 
 extern "C" int hilberta_plan_destroy(hilberta_plan_t *plan) {
