@@ -203,6 +203,14 @@ int hilberta_forward_host(const void *q, const void *k, const void *v, void *out
  * device.  Clears the flag. */
 int hilberta_plan_status(hilberta_plan_t *plan);
 
+/* Failure-detection self-test: launches a one-warp kernel that waits, with a 1 ms
+ * deadline, on a barrier nothing arrives on -- the same bounded wait every role of
+ * the attention kernel uses -- so that the wait expires, the status words of `plan` are
+ * written and the kernel returns normally.  After it, hilberta_plan_status(plan) must
+ * return HILBERTA_ERR_TIMEOUT once and the device must stay usable.  Asynchronous on
+ * `stream`. */
+int hilberta_selftest_timeout(hilberta_plan_t *plan, void *stream);
+
 /* Number of kernels the library has launched in this process (all entry points). */
 uint64_t hilberta_launch_count(void);
 

@@ -28,7 +28,7 @@ SYMBOLS = (
     "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_lse", "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
-    "hilberta_plan_status", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
+    "hilberta_plan_status", "hilberta_selftest_timeout", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
     "hilberta_last_cuda_error",
 )
 
@@ -77,6 +77,8 @@ def lib():
         f = getattr(L, name)
         f.argtypes = [vp, vp, vp, i32, i32, i32, vp]
         f.restype = i32
+    L.hilberta_selftest_timeout.argtypes = [vp, vp]
+    L.hilberta_selftest_timeout.restype = i32
     L.hilberta_plan_status.argtypes = [vp]
     L.hilberta_plan_status.restype = i32
     L.hilberta_launch_count.argtypes = []

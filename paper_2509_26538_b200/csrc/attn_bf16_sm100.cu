@@ -88,14 +88,14 @@ struct Params {
 
 // Wait with a deadline; on expiry record where and raise the CTA's abort flag.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                              int *status, int code) {
+                                              int *status, int code, long long limit = WAIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63) == 63) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_CYCLES) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0, code) == 0) {
                     status[1] = blockIdx.x;
@@ -541,6 +541,21 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
 }
 
+// Exercises the bounded wait on purpose: one warp waits, with a 1 ms deadline, on a
+// barrier that nothing ever arrives on, records the expiry like the attention kernel
+// does and returns normally.  Used by hilberta_selftest_timeout.
+__global__ void timeout_probe_kernel(int *status) {
+    __shared__ uint64_t never;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&never), 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    wait_or_abort(smem_u32(&never), 0, &abort_flag, status, 0x7e57, 2000000ll);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -597,6 +612,12 @@ void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, cons
 }
 
 }  // namespace
+
+int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
+    timeout_probe_kernel<<<1, 32, 0, stream>>>(p->d_status);
+    HB_LAUNCHED();
+    return HILBERTA_OK;
+}
 
 // Work list: prefix rows read the whole sequence; the rows of each slid tile
 // read the prefix and the tile's own one or two ranges.  Longest items first.

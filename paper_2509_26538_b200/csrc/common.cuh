@@ -101,4 +101,5 @@ int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, con
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
                      float *lse, const int *out_map, cudaStream_t stream);
 int attn_bf16_prepare(hilberta_plan_t *p);
+int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream);
 }  // namespace hilberta

@@ -535,6 +535,11 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
     return HILBERTA_OK;
 }
 
+extern "C" int hilberta_selftest_timeout(hilberta_plan_t *p, void *stream) {
+    if (!p) return HILBERTA_ERR_INVALID;
+    return launch_timeout_probe(p, (cudaStream_t)stream);
+}
+
 extern "C" int hilberta_plan_status(hilberta_plan_t *p) {
     if (!p) return HILBERTA_ERR_INVALID;
     int h[4] = {0, 0, 0, 0};
