@@ -201,6 +201,7 @@ def main():
     ap.add_argument("--shared", type=int, default=-1, help="override the side of the central shared region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the dense / SDPA context rows")
     ap.add_argument("--schedule", action="store_true",
                     help="also time the 57-layer per-step schedule (one permute, 57 forwards with the "
                          "per-layer offsets, one unpermute) on the chosen workload's shape")
@@ -342,6 +343,41 @@ def main():
                "steps": n_e2e}
         assert torch.isfinite(oh.float()).all()
 
+    # ---- context rows (not part of the metric): dense attention of this build and PyTorch SDPA
+    context_rows = None
+    if world == 1 and not args.no_context:
+        def timed(fn, n=5):
+            fn()
+            torch.cuda.synchronize()
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(n):
+                fn()
+            b_.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b_) / n
+        dense_flops = 4.0 * wl.head_dim * wl.heads * wl.batch * wl.S * wl.S
+        context_rows = {"dense_gflop": dense_flops / 1e9}
+        try:
+            n_pad = 1
+            while n_pad < max(wl.H, wl.W):
+                n_pad *= 2
+            dense = hb.Plan(wl.H, wl.W, n_pad * n_pad, 0, 0, wl.n_text)   # one tile, no shared region: every pair kept
+            dense.bind_like(qp)
+            ms = timed(lambda: dense.forward(qp, kp, vp, op))
+            assert dense.status() == 0
+            dense.destroy()
+            context_rows["dense_this_build"] = {"ms": ms, "tflops": dense_flops / (ms * 1e-3) / 1e12}
+        except Exception as e:  # context only
+            context_rows["dense_this_build"] = {"error": str(e)[:120]}
+        try:
+            ms = timed(lambda: torch.nn.functional.scaled_dot_product_attention(qp, kp, vp))
+            context_rows["torch_sdpa_dense_bf16"] = {"ms": ms, "tflops": dense_flops / (ms * 1e-3) / 1e12}
+        except Exception as e:
+            context_rows["torch_sdpa_dense_bf16"] = {"error": str(e)[:120]}
+        context_rows["sparse_speedup_vs_dense_this_build"] = (
+            context_rows["dense_this_build"]["ms"] / fwd_avg if "ms" in context_rows["dense_this_build"] else None)
+
     schedule = None
     if args.schedule:
         from paper_2509_26538_b200.inputs import SCHEDULE_LAYERS, schedule_offset
@@ -408,7 +444,7 @@ def main():
                      "traffic": FORWARD_DRAM_TRAFFIC_BYTES.get(wl.name)},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "schedule57": schedule,
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
-                             "(4.36 ms per call at 2048^2, 16 tiles)"},
+                             "(4.36 ms per call at 2048^2, 16 tiles)", "same_gpu": context_rows},
     }
     if not args.no_cpu_baseline and world == 1 and not args.groups:
         tf, threads, desc, dt = oracle_sample(wl, 15.0)
