@@ -12,7 +12,8 @@
  *   - All functions return an int status: 0 on success, a negative
  *     HILBERTA_ERR_* code otherwise.  Nothing throws or aborts.
  *   - "device pointer" = memory of the CUDA device that was current when the
- *     plan was created; "host pointer" = ordinary host memory.
+ *     plan was created; "host pointer" = ordinary host memory.  Calls that launch
+ *     kernels return ERR_INVALID if another device is current.
  *   - `stream` arguments are a cudaStream_t passed as void* (NULL = default
  *     stream).
  *   - ORIGINAL token order:  [ text 0..n_text ) ++ [ image tokens row-major,

@@ -473,6 +473,9 @@ static int forward_impl(const void *q, const void *k, const void *v, void *out, 
     if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
     if (out == q || out == k || out == v) return HILBERTA_ERR_INVALID;
+    int dev = -1;
+    HB_CUDA(cudaGetDevice(&dev));
+    if (dev != p->device) return HILBERTA_ERR_INVALID;  // the plan's tables live on another device
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == HILBERTA_FP32) return launch_attn_fp32(p, q, k, v, out, lse, out_map, st);
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
