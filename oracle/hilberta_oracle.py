@@ -27,6 +27,8 @@ Where each piece comes from
   text tokens are treated exactly like the shared anchor region).
 * attention : softmax(s * q k^T restricted to the mask) v, the quantity
   Algorithm 1's online softmax reaches up to rounding.
+* attention_backward : the derivative of that quantity (the paper fine-tunes
+  through its kernel, Sec. 4.1, without printing the backward pass).
 * token_classes_compact / mask_compact / plan_arrays_compact : Appendix A read
   literally (Algorithm 1's S = N / G over the non-shared tokens).
 * plan arrays : the memory layout of Appendix A (prefix of text + shared
@@ -37,7 +39,9 @@ Pins (tests/test_oracle_*.py): bijection, 4-neighbour steps, aligned-block
 squares, mirror law, an independent bit-pair construction, hand-derived 4x4 and
 8x8 tables, mask symmetry/diagonal/row counts, the ERF law, periodicity in the
 offset, reduction to dense attention (checked against torch SDPA in fp64), the
-block-diagonal case, brute-force masks on tiny grids, Table 1's GFLOPs column.
+block-diagonal case, brute-force masks on tiny grids, Table 1's GFLOPs column;
+attention_backward: central finite differences of attention(), torch autograd in
+fp64, and the identities sum_j dK_j = 0 and sum_j dV_j = sum_i dO_i.
 """
 from __future__ import annotations
 
@@ -256,6 +260,42 @@ def attention_rows(q, k, v, is_global, group, rows, scale=None):
                 p = np.exp(logits - logits.max())
                 out[b, h, n] = (p @ vv) / p.sum()
     return out
+
+
+def attention_backward(q, k, v, M, dout, scale=None):
+    """Gradients of  L = sum(O * dout)  with  O = attention(q, k, v, M), in float64.
+
+    The paper trains through its kernel (Sec. 4.1, LoRA fine-tuning) but prints
+    no backward formulas, so this is the plain derivative of the definition
+    above, written out per (batch, head) with dense S x S matrices:
+
+        P   = softmax over the allowed keys of  scale * Q K^T
+        dV  = P^T dO
+        dP  = dO V^T
+        dS  = P * (dP - rowsum(P * dP))          (zero where M is zero)
+        dQ  = scale * dS K,      dK = scale * dS^T Q
+
+    Returns (dq, dk, dv), each [B, heads, S, D].
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    dout = np.asarray(dout, dtype=np.float64)
+    B, Hh, S, D = q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    dq, dk, dv = np.empty_like(q), np.empty_like(k), np.empty_like(v)
+    for b in range(B):
+        for h in range(Hh):
+            logits = np.where(M, scale * (q[b, h] @ k[b, h].T), -np.inf)
+            p = np.exp(logits - logits.max(axis=1, keepdims=True))
+            p /= p.sum(axis=1, keepdims=True)
+            dp = dout[b, h] @ v[b, h].T
+            ds = p * (dp - (p * dp).sum(axis=1, keepdims=True))
+            dv[b, h] = p.T @ dout[b, h]
+            dq[b, h] = scale * (ds @ k[b, h])
+            dk[b, h] = scale * (ds.T @ q[b, h])
+    return dq, dk, dv
 
 
 # --------------------------------------------------------------------------
