@@ -164,6 +164,33 @@ int hilberta_forward(const void *q, const void *k, const void *v, void *out,
 int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out, float *lse,
                          const hilberta_plan_t *plan, void *stream);
 
+/* Backward pass of hilberta_forward: the gradients of  sum(out * dout)  with
+ * respect to q, k and v.  The paper fine-tunes through its kernel (Sec. 4.1, LoRA)
+ * but does not describe the backward pass; this is the derivative of Algorithm 1's
+ * result under the same mask, layout and plan:
+ *     P = exp(scale * q k^T - lse) on kept pairs,   dP = dout v^T,
+ *     delta_i = sum_d dout[i, d] * out[i, d],       dS = P * (dP - delta),
+ *     dq = scale * dS k,    dk = scale * dS^T q,    dv = P^T dout.
+ *
+ * dout, q, k, v, out : device pointers, PHYSICAL order, bf16, the bound shape and
+ *                      strides; `out` and `lse` are what hilberta_forward_lse wrote
+ *                      for these q, k, v.
+ * lse                : device pointer, [batch * heads, S] fp32 (natural log).
+ * dq, dk, dv         : device pointers, written; same shape and strides as q; must
+ *                      not alias each other or any input.  Every row is written.
+ * All pointers 16-byte aligned (lse: 4).  Asynchronous on `stream`; three kernel
+ * launches; no allocation, no synchronisation.  A per-row scratch array
+ * (batch * heads * S floats, owned by the plan, allocated by hilberta_plan_bind)
+ * carries delta between the launches, so two backward calls on the same plan
+ * must not overlap on the device.
+ *
+ * Errors: ERR_INVALID (NULL, misaligned or aliasing pointers, wrong device),
+ * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding: only the bf16 tensor-core path has a
+ * backward pass), ERR_CUDA. */
+int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
+                      const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
+                      void *stream);
+
 /* hilberta_forward with the exit gather of Sec. 3.4 fused into its epilogue (the
  * last attention layer of a step): q, k, v are in PHYSICAL order as for
  * hilberta_forward; `out` is written in ORIGINAL token order, i.e. physical row p

@@ -25,7 +25,8 @@ BF16, FP32 = 0, 1
 SYMBOLS = (
     "hilberta_plan", "hilberta_plan_groups", "hilberta_plan_destroy", "hilberta_plan_export",
     "hilberta_plan_bind",
-    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_lse", "hilberta_permute",
+    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_lse", "hilberta_backward",
+    "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
     "hilberta_plan_status", "hilberta_selftest_timeout", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
@@ -71,6 +72,8 @@ def lib():
     L.hilberta_forward_unpermute.restype = i32
     L.hilberta_forward_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_lse.restype = i32
+    L.hilberta_backward.argtypes = [vp] * 11
+    L.hilberta_backward.restype = i32
     L.hilberta_forward_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_host.restype = i32
     for name in ("hilberta_permute", "hilberta_unpermute"):
@@ -194,6 +197,13 @@ class Plan:
         _check(lib().hilberta_forward_lse(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                           lse.data_ptr(), self._h, _stream_ptr(stream)), "hilberta_forward_lse")
         return out, lse
+
+    def backward(self, dout, q, k, v, out, lse, dq, dk, dv, stream=None):
+        """dq, dk, dv from dout and the forward's inputs, output and lse (all physical order, bf16)."""
+        _check(lib().hilberta_backward(dout.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                       lse.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), self._h,
+                                       _stream_ptr(stream)), "hilberta_backward")
+        return dq, dk, dv
 
     def forward_host(self, q, k, v, out, stream=None):
         """q, k, v, out: HOST tensors (pinned for asynchronous copies), original order."""

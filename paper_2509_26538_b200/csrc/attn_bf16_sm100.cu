@@ -50,7 +50,6 @@ constexpr int SLAB_BYTES = TILE_BYTES / 2;
 constexpr int THREADS = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle (register donors)
 constexpr int SMEM_BYTES = (QT + NSTAGE) * TILE_BYTES + 1024;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr long long WAIT_CYCLES = 2000000000ll;  // ~1 s: far beyond any legitimate wait
 constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 #ifndef HB_POLY_MASK
 #define HB_POLY_MASK 3   // pair i of every 16 runs its two exponentials on the FMA pipes when (i & MASK) == MASK (3: one pair in four); 0xff = never
@@ -86,35 +85,8 @@ struct Params {
     int *status;
 };
 
-// Wait with a deadline; on expiry record where and raise the CTA's abort flag.
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                              int *status, int code, long long limit = WAIT_CYCLES) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t i = 0;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63) == 63) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit) {
-                *abort_flag = 1;
-                if (atomicCAS(status, 0, code) == 0) {
-                    status[1] = blockIdx.x;
-                    status[2] = (int)parity;
-                }
-                return false;
-            }
-        }
-    }
-}
-
 __device__ __forceinline__ int item_blocks(const WorkItem &it, int seg) {
     return (it.seg_len[seg] + BN - 1) / BN;
-}
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -140,17 +112,6 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
     p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
     p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
     return p;
-}
-
-__device__ __forceinline__ void st_global_v8(void *p, const uint32_t *w) {
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
-                 : "memory");
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&h);
 }
 
 // S_t = Q_t K^T for one 128-key block: 8 MMAs of K = 16.
@@ -574,13 +535,15 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [batch, heads, S, 128] bf16 with element strides -> 4-D map, box = 64 columns x 128 rows.
-int make_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p) {
+}  // namespace
+
+// [batch, heads, S, 128] bf16 with element strides -> 4-D map, box = 64 columns x box_rows rows.
+int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, int box_rows) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return HILBERTA_ERR_CUDA;
-    cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)p->S, (cuuint64_t)p->heads, (cuuint64_t)p->batch};
+    cuuint64_t dims[4] = {128, (cuuint64_t)p->S, (cuuint64_t)p->heads, (cuuint64_t)p->batch};
     cuuint64_t strides[3] = {(cuuint64_t)p->stride_s * 2, (cuuint64_t)p->stride_h * 2, (cuuint64_t)p->stride_b * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)BN, 1, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -591,6 +554,8 @@ int make_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p) {
     }
     return HILBERTA_OK;
 }
+
+namespace {
 
 void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, const int *seg_start,
                const int *seg_len) {
@@ -696,9 +661,9 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     if (p->n_work == 0) return HILBERTA_OK;
     CUtensorMap mq, mk, mv;
     int rc;
-    if ((rc = make_map(&mq, q, p)) != HILBERTA_OK) return rc;
-    if ((rc = make_map(&mk, k, p)) != HILBERTA_OK) return rc;
-    if ((rc = make_map(&mv, v, p)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mq, q, p, BN)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mk, k, p, BN)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mv, v, p, BN)) != HILBERTA_OK) return rc;
     Params prm;
     prm.work = p->d_work;
     prm.units = p->d_units;

@@ -84,6 +84,14 @@ struct hilberta_plan_s {
     hilberta::WorkUnit *d_units;  // [n_work * batch * heads], grouped by CTA
     int *d_cta_begin;             // [n_cta + 1]
     int n_cta;
+    // backward pass: 128-row items over the same key lists, their schedule, and the
+    // per-row scratch delta = rowsum(dO * O) that both backward kernels read
+    hilberta::WorkItem *d_bwd_work;
+    int n_bwd_work;
+    hilberta::WorkUnit *d_bwd_units;
+    int *d_bwd_cta_begin;
+    int n_bwd_cta;
+    float *d_delta;               // [batch * heads * S]
     int *d_status;  // [4] error word + diagnostics written by bounded waits
     // workspace of hilberta_forward_host
     void *ws;
@@ -101,5 +109,10 @@ int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, con
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
                      float *lse, const int *out_map, cudaStream_t stream);
 int attn_bf16_prepare(hilberta_plan_t *p);
+int attn_bwd_prepare(hilberta_plan_t *p);
+// dq, dk, dv (bf16, physical order, the bound strides) from dout, q, k, v, out and the forward's lse.
+int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, const void *k, const void *v,
+                    const void *out, const float *lse, void *dq, void *dk, void *dv, float *delta,
+                    cudaStream_t stream);
 int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream);
 }  // namespace hilberta

@@ -208,6 +208,10 @@ static void free_plan(hilberta_plan_t *p) {
     cudaFree(p->d_work);
     cudaFree(p->d_units);
     cudaFree(p->d_cta_begin);
+    cudaFree(p->d_bwd_work);
+    cudaFree(p->d_bwd_units);
+    cudaFree(p->d_bwd_cta_begin);
+    cudaFree(p->d_delta);
     cudaFree(p->d_status);
     cudaFree(p->ws);
     delete p;
@@ -463,6 +467,8 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
     if (dtype == HILBERTA_BF16) {
         int rc = attn_bf16_prepare(p);
         if (rc != HILBERTA_OK) return rc;
+        rc = attn_bwd_prepare(p);
+        if (rc != HILBERTA_OK) return rc;
     }
     p->bound = true;
     return HILBERTA_OK;
@@ -497,6 +503,30 @@ extern "C" int hilberta_forward_lse(const void *q, const void *k, const void *v,
                                     const hilberta_plan_t *p, void *stream) {
     if (!lse || ((uintptr_t)lse & 3)) return HILBERTA_ERR_INVALID;
     return forward_impl(q, k, v, out, lse, p, nullptr, stream);
+}
+
+extern "C" int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
+                                 const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *p,
+                                 void *stream) {
+    if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
+    if (!p->bound) return HILBERTA_ERR_UNBOUND;
+    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
+    const void *in[5] = {dout, q, k, v, out};
+    void *outs[3] = {dq, dk, dv};
+    uintptr_t bits = (uintptr_t)lse & 3 ? 15 : 0;
+    for (int i = 0; i < 3; ++i) {
+        bits |= (uintptr_t)outs[i];
+        for (int j = 0; j < 5; ++j)
+            if (outs[i] == in[j]) return HILBERTA_ERR_INVALID;
+        for (int j = 0; j < i; ++j)
+            if (outs[i] == outs[j]) return HILBERTA_ERR_INVALID;
+    }
+    for (int j = 0; j < 5; ++j) bits |= (uintptr_t)in[j];
+    if (bits & 15) return HILBERTA_ERR_INVALID;
+    int dev = -1;
+    HB_CUDA(cudaGetDevice(&dev));
+    if (dev != p->device) return HILBERTA_ERR_INVALID;
+    return launch_attn_bwd(p, dout, q, k, v, out, lse, dq, dk, dv, p->d_delta, (cudaStream_t)stream);
 }
 
 // Whole path for host-resident activations: H2D copies, three entry gathers,

@@ -1,0 +1,112 @@
+"""Backward pass (dq, dk, dv) through the C ABI against the fp64 oracle.
+
+Tolerances.  Everything the kernel rounds is rounded to bf16 (relative step 2^-9,
+rms 2^-9 / sqrt(3) = 1.1e-3): the stored gradients, the weights P and the logit
+gradients dS that feed the tensor cores, and the forward output O that enters
+delta.  These are independent, so the relative L2 error is about sqrt(3) * 1.1e-3
+= 2e-3 (measured 2.3e-3 to 2.4e-3); the bar is the forward's 5e-3, and max-abs is
+1e-2 of the gradient's scale.  Near-one-hot rows ("peaky" inputs) cancel
+dP - delta almost completely, which amplifies the rounding of O; those cases get
+twice the bars.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attn_c
+from oracle import hilberta_oracle as orc
+from paper_2509_26538_b200 import binding as hb
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(H, W, tile, o, hs, nt, B, heads, groups=0, q_gain=1.0, seed=5):
+    S = nt + H * W
+    g = torch.Generator().manual_seed(seed)
+    q, k, v, do = (torch.randn((B, heads, S, 128), generator=g) for _ in range(4))
+    q, k, v, do = ((q * q_gain).to(torch.bfloat16), k.to(torch.bfloat16), v.to(torch.bfloat16),
+                   do.to(torch.bfloat16))
+    if groups:
+        ig, grp = orc.token_classes_compact(H, W, groups, o, hs, nt)
+    else:
+        ig, grp = orc.token_classes(H, W, tile, o, hs, nt)
+    ref = attn_c.attention_backward(q.float().numpy(), k.float().numpy(), v.float().numpy(), do.float().numpy(),
+                                    ig, grp)
+    plan = hb.Plan(H, W, tile, o, hs, nt, groups=groups)
+    try:
+        p2o = torch.from_numpy(plan.export(hb.EXPORT_PHYS2ORIG).astype(np.int64))
+        qp, kp, vp, dop = (t[:, :, p2o].contiguous().cuda() for t in (q, k, v, do))
+        out = torch.empty_like(qp)
+        lse = torch.empty((B, heads, S), device="cuda", dtype=torch.float32)
+        plan.bind_like(qp)
+        plan.forward_lse(qp, kp, vp, out, lse)
+        grads = [torch.full_like(qp, float("nan")) for _ in range(3)]
+        plan.backward(dop, qp, kp, vp, out, lse, *grads)
+        again = [torch.empty_like(qp) for _ in range(3)]
+        plan.backward(dop, qp, kp, vp, out, lse, *again)
+        assert plan.status() == 0
+        for a, b in zip(grads, again):
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))  # no atomics: bit-reproducible
+        got = []
+        for t in grads:
+            full = torch.empty((B, heads, S, 128), dtype=torch.float64)
+            full[:, :, p2o] = t.cpu().double()
+            got.append(full.numpy())
+    finally:
+        plan.destroy()
+    return got, ref
+
+
+@pytest.mark.parametrize("H,W,tile,o,hs,nt,B,heads,groups", [
+    (16, 16, 64, 16, 2, 0, 1, 1, 0),        # four tiles, no text, ragged tile ranges
+    (16, 16, 64, 16, 2, 40, 2, 2, 0),       # text prefix, batch 2
+    (32, 32, 256, 128, 4, 77, 1, 2, 0),     # several 128-row items per tile, wrapped tile
+    (24, 40, 256, 100, 4, 33, 1, 2, 0),     # non-square grid on the padded curve
+    (16, 16, 256, 0, 0, 0, 1, 2, 0),        # one tile, no shared region: dense attention
+    (32, 32, 0, 37, 4, 50, 1, 2, 6),        # equal groups over the non-shared tokens (Appendix A)
+    (16, 16, 64, 0, 16, 3, 1, 1, 0),        # every image token shared: prefix rows only
+])
+def test_backward_matches_oracle(H, W, tile, o, hs, nt, B, heads, groups):
+    got, ref = _run(H, W, tile, o, hs, nt, B, heads, groups)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert np.isfinite(g).all(), name
+        assert orc.rel_l2_err(g, r) <= 5e-3, (name, orc.rel_l2_err(g, r))
+        assert orc.max_abs_err(g, r) <= 1e-2 * max(1.0, np.abs(r).max()), (name, orc.max_abs_err(g, r))
+
+
+def test_backward_flux1024_two_heads():
+    got, ref = _run(64, 64, 1024, 512, 8, 512, 1, 2)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert orc.rel_l2_err(g, r) <= 5e-3, (name, orc.rel_l2_err(g, r))
+        assert orc.max_abs_err(g, r) <= 1e-2 * max(1.0, np.abs(r).max()), name
+
+
+def test_backward_peaky_inputs():
+    got, ref = _run(32, 32, 256, 128, 4, 77, 1, 2, q_gain=8.0)
+    for name, g, r in zip(("dq", "dk", "dv"), got, ref):
+        assert np.isfinite(g).all(), name
+        assert orc.rel_l2_err(g, r) <= 1e-2, (name, orc.rel_l2_err(g, r))
+        assert orc.max_abs_err(g, r) <= 2e-2 * max(1.0, np.abs(r).max()), name
+
+
+def test_backward_argument_checks():
+    plan = hb.Plan(16, 16, 64, 0, 2, 0)
+    try:
+        x = torch.zeros((1, 1, 256, 128), device="cuda", dtype=torch.bfloat16)
+        bufs = [torch.zeros_like(x) for _ in range(8)]
+        lse = torch.zeros((1, 1, 256), device="cuda", dtype=torch.float32)
+        ptr = [t.data_ptr() for t in bufs]
+        L = hb.lib()
+        assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), *ptr[5:8], plan._h, None) == hb.ERR_UNBOUND
+        plan.bind_like(x)
+        assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), *ptr[5:8], plan._h, None) == hb.OK
+        assert L.hilberta_backward(*ptr[:5], None, *ptr[5:8], plan._h, None) == hb.ERR_INVALID
+        assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), ptr[5], ptr[5], ptr[7], plan._h, None) == hb.ERR_INVALID
+        assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), ptr[1], ptr[6], ptr[7], plan._h, None) == hb.ERR_INVALID
+        assert L.hilberta_backward(ptr[0] + 2, *ptr[1:5], lse.data_ptr(), *ptr[5:8], plan._h, None) == hb.ERR_INVALID
+        assert plan.status() == 0
+        f = torch.zeros((1, 1, 256, 64), device="cuda", dtype=torch.float32)
+        plan.bind_like(f)
+        assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), *ptr[5:8], plan._h, None) == hb.ERR_UNSUPPORTED
+    finally:
+        plan.destroy()
