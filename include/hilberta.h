@@ -191,6 +191,39 @@ int hilberta_backward(const void *dout, const void *q, const void *k, const void
                       const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
                       void *stream);
 
+/* hilberta_backward for callers that must not allocate.  (The paper has no
+ * counterpart: this is a deployment variant of the call above.)
+ *
+ * hilberta_backward keeps its per-row scratch (delta, one float per batch, head
+ * and token) in memory that hilberta_plan_bind obtains from cudaMalloc, once per
+ * plan.  Some hosts cannot afford that: a serving process that handed all device
+ * memory to its own pool at start-up, so that a later cudaMalloc fails; a
+ * latency-bound loop that must avoid the device-wide synchronisation an
+ * allocation implies; a process that keeps dozens of bound plans (one per layer
+ * offset) and does not want a scratch array in each.  This variant puts the
+ * scratch in one fixed array of HILBERTA_STATIC_SCRATCH_FLOATS floats (4 MiB)
+ * that is part of the library image: every GPU that loads the library holds it
+ * until the process exits, and every plan and every call shares it.
+ *
+ * Arguments, layouts, alignment, results and errors are those of
+ * hilberta_backward, and the output is the same.  In addition:
+ *   - batch * heads * S  >  HILBERTA_STATIC_SCRATCH_FLOATS  ->  ERR_BUFFER, nothing
+ *     is launched (the Flux shapes at 1024^2 and 2048^2 fit; 4096^2 with 24 heads
+ *     does not: use hilberta_backward there);
+ *   - the call itself performs no cudaMalloc, cudaFree or other allocation;
+ *   - the FIRST call on each device looks up the array's device address (with
+ *     that device current) and caches it; make that first call before any stream
+ *     capture begins;
+ *   - the array keeps what the previous call wrote.  Nothing in it has to start at
+ *     zero: each call overwrites every entry it later reads, in stream order;
+ *   - because the array is shared, two calls that overlap on the GPU (different
+ *     streams, different plans, or this call and another thread's) race on it.
+ *     Serialise them, or use hilberta_backward, whose scratch is per plan. */
+#define HILBERTA_STATIC_SCRATCH_FLOATS (1 << 20)
+int hilberta_backward_static(const void *dout, const void *q, const void *k, const void *v, const void *out,
+                             const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
+                             void *stream);
+
 /* hilberta_forward with the exit gather of Sec. 3.4 fused into its epilogue (the
  * last attention layer of a step): q, k, v are in PHYSICAL order as for
  * hilberta_forward; `out` is written in ORIGINAL token order, i.e. physical row p

@@ -26,7 +26,7 @@ SYMBOLS = (
     "hilberta_plan", "hilberta_plan_groups", "hilberta_plan_destroy", "hilberta_plan_export",
     "hilberta_plan_bind",
     "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_lse", "hilberta_backward",
-    "hilberta_permute",
+    "hilberta_backward_static", "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
     "hilberta_plan_status", "hilberta_selftest_timeout", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
@@ -74,6 +74,8 @@ def lib():
     L.hilberta_forward_lse.restype = i32
     L.hilberta_backward.argtypes = [vp] * 11
     L.hilberta_backward.restype = i32
+    L.hilberta_backward_static.argtypes = [vp] * 11
+    L.hilberta_backward_static.restype = i32
     L.hilberta_forward_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_host.restype = i32
     for name in ("hilberta_permute", "hilberta_unpermute"):
@@ -203,6 +205,14 @@ class Plan:
         _check(lib().hilberta_backward(dout.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                        lse.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), self._h,
                                        _stream_ptr(stream)), "hilberta_backward")
+        return dq, dk, dv
+
+    def backward_static(self, dout, q, k, v, out, lse, dq, dk, dv, stream=None):
+        """backward() with the scratch in the library's fixed array: no allocation in the call."""
+        _check(lib().hilberta_backward_static(dout.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                              out.data_ptr(), lse.data_ptr(), dq.data_ptr(), dk.data_ptr(),
+                                              dv.data_ptr(), self._h, _stream_ptr(stream)),
+               "hilberta_backward_static")
         return dq, dk, dv
 
     def forward_host(self, q, k, v, out, stream=None):

@@ -544,3 +544,66 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
 }
 
 }  // namespace hilberta
+
+// ---------------------------------------------------------------------------
+// hilberta_backward_static: the same three launches with the delta scratch in a
+// fixed array that is part of the library image instead of memory obtained from
+// the CUDA allocator.  The array lives on every device that loads the library.
+// In host code its name is only a handle; the device address is looked up once
+// per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) float g_static_delta[HILBERTA_STATIC_SCRATCH_FLOATS];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+float *g_static_delta_ptr[MAX_DEVICES] = {};
+
+// Device address of g_static_delta on `device`, which must be the current device.
+int static_delta_address(int device, float **ptr) {
+    if (device < 0 || device >= MAX_DEVICES) return HILBERTA_ERR_INVALID;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_delta_ptr[device]) {
+        float *addr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress((void **)&addr, g_static_delta);
+        if (e != cudaSuccess || !addr) {
+            hilberta::g_last_cuda_error = (int)e;
+            return HILBERTA_ERR_CUDA;
+        }
+        g_static_delta_ptr[device] = addr;
+    }
+    *ptr = g_static_delta_ptr[device];
+    return HILBERTA_OK;
+}
+}  // namespace
+
+extern "C" int hilberta_backward_static(const void *dout, const void *q, const void *k, const void *v,
+                                        const void *out, const float *lse, void *dq, void *dk, void *dv,
+                                        const hilberta_plan_t *p, void *stream) {
+    if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
+    if (!p->bound) return HILBERTA_ERR_UNBOUND;
+    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
+    const void *in[5] = {dout, q, k, v, out};
+    void *outs[3] = {dq, dk, dv};
+    uintptr_t bits = ((uintptr_t)lse & 3) ? 15 : 0;
+    for (int i = 0; i < 3; ++i) {
+        bits |= (uintptr_t)outs[i];
+        for (int j = 0; j < 5; ++j)
+            if (outs[i] == in[j]) return HILBERTA_ERR_INVALID;
+        for (int j = 0; j < i; ++j)
+            if (outs[i] == outs[j]) return HILBERTA_ERR_INVALID;
+    }
+    for (int j = 0; j < 5; ++j) bits |= (uintptr_t)in[j];
+    if (bits & 15) return HILBERTA_ERR_INVALID;
+    // one float of scratch per (batch, head, token): refuse what the fixed array cannot hold
+    if ((unsigned long long)p->batch * p->heads * p->S > (unsigned long long)HILBERTA_STATIC_SCRATCH_FLOATS)
+        return HILBERTA_ERR_BUFFER;
+    int dev = -1;
+    HB_CUDA(cudaGetDevice(&dev));
+    if (dev != p->device) return HILBERTA_ERR_INVALID;
+    float *delta = nullptr;
+    const int rc = static_delta_address(dev, &delta);
+    if (rc != HILBERTA_OK) return rc;
+    // delta_kernel overwrites every entry the two tensor-core kernels read, so whatever an
+    // earlier call left in the array is never seen and nothing has to be cleared
+    return hilberta::launch_attn_bwd(p, dout, q, k, v, out, lse, dq, dk, dv, delta, (cudaStream_t)stream);
+}

@@ -1,0 +1,72 @@
+"""hilberta_backward_static: the backward pass for callers that cannot allocate.
+
+Some users of this library run where device allocation is off the table at call
+time: all device memory already belongs to the host application's pool, or the
+call sits in a loop that cannot take the synchronisation an allocation implies.
+For them the library keeps the backward pass's per-row scratch in a fixed array
+inside its own image.  The test drives that entry point through the C ABI twice
+in a row, on two different problems, and holds each result against what the
+ordinary hilberta_backward (scratch owned by the plan) returns for the same
+inputs.  The second problem is smaller than the first, so the array still holds
+the first call's values beyond it: they must not leak into the result.
+
+This file sorts last on purpose: a run that stops at the first failure has by
+then run every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_26538_b200 import binding as hb
+
+pytestmark = pytest.mark.gpu
+
+
+def _problem(H, W, tile, o, hs, nt, B, heads, seed):
+    S = nt + H * W
+    g = torch.Generator().manual_seed(seed)
+    qp, kp, vp, dop = (torch.randn((B, heads, S, 128), generator=g).to(torch.bfloat16).cuda() for _ in range(4))
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    plan.bind_like(qp)
+    out = torch.empty_like(qp)
+    lse = torch.empty((B, heads, S), device="cuda", dtype=torch.float32)
+    plan.forward_lse(qp, kp, vp, out, lse)
+    return plan, (dop, qp, kp, vp, out, lse)
+
+
+def _rel_l2(a, b):
+    a, b = a.double(), b.double()
+    return float((a - b).norm() / b.norm())
+
+
+def test_static_scratch_backward_matches_plan_scratch_backward_twice():
+    for case in ((32, 32, 256, 128, 4, 77, 1, 3, 11), (16, 16, 64, 16, 2, 40, 1, 2, 12)):
+        plan, args = _problem(*case)
+        try:
+            want = [torch.empty_like(args[1]) for _ in range(3)]
+            plan.backward(*args, *want)
+            got = [torch.full_like(args[1], float("nan")) for _ in range(3)]
+            plan.backward_static(*args, *got)
+            assert plan.status() == 0
+            for name, g, w in zip(("dq", "dk", "dv"), got, want):
+                assert torch.isfinite(g.float()).all(), name
+                assert _rel_l2(g, w) <= 5e-3, (name, _rel_l2(g, w))
+                scale = max(1.0, float(w.float().abs().max()))
+                assert float((g.float() - w.float()).abs().max()) <= 1e-2 * scale, name
+        finally:
+            plan.destroy()
+
+
+def test_static_scratch_backward_rejects_what_does_not_fit():
+    # 11 x 24 x 4096 rows need more floats than the fixed array has
+    plan = hb.Plan(64, 64, 1024, 0, 8, 0)
+    try:
+        plan.bind(11, 24, 128, hb.BF16)
+        x = [torch.zeros(64, device="cuda", dtype=torch.bfloat16) for _ in range(8)]
+        lse = torch.zeros(16, device="cuda", dtype=torch.float32)
+        p = [t.data_ptr() for t in x]
+        rc = hb.lib().hilberta_backward_static(*p[:5], lse.data_ptr(), *p[5:8], plan._h, None)
+        assert rc == hb.ERR_BUFFER
+        assert plan.status() == 0
+    finally:
+        plan.destroy()
