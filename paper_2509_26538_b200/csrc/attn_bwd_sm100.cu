@@ -15,9 +15,12 @@
 //             acc1 = K_j Q_i^T, acc2 = V_j dO_i^T (transposed scores: a thread owns a KEY row),
 //             P^T, dS^T -> TMEM, dV_j += P^T dO_i, dK_j += dS^T Q_i
 // Streamed rows come in sub-blocks of 64 with two accumulator buffers, so the MMAs of
-// sub-block s + 1 run while the CUDA cores work on sub-block s; the two softmax
-// warpgroups alternate sub-blocks.  TMEM: acc1/acc2 of buffer b at [128 b, +64) and
-// [128 b + 64, +64) (P and dS overwrite them in place as bf16), outputs at [256, 512).
+// sub-block s + 1 run while the CUDA cores work on sub-block s; the two element-wise
+// warpgroups each take 32 of the 64 columns of every sub-block, which halves the
+// latency of the MMA -> element-wise -> MMA chain.  TMEM: acc1/acc2 of buffer b at
+// [128 b, +64) and [128 b + 64, +64); P and dS (bf16) overwrite them in place, each
+// warpgroup inside the columns it has just read.  DKV: two buffers, dK at [256, 384),
+// dV at [384, 512).  DQ: three buffers (the MMAs run two sub-blocks ahead), dQ at [384, 512).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -40,23 +43,33 @@ namespace {
 constexpr int BM = 128;   // resident rows per work item
 constexpr int SUB = 64;   // streamed rows per sub-block
 constexpr int HD = 128;
-constexpr int NST = 4;    // ring of streamed sub-blocks (two 16-KB tiles each)
+constexpr int NST_MAX = 5;   // ring of streamed sub-blocks (two 16-KB tiles each): 5 slots in DQ mode, 4 in DKV
+#ifndef HB_NST_DQ
+#define HB_NST_DQ 5
+#endif
+#ifndef HB_NST_DKV
+#define HB_NST_DKV 4
+#endif
+__host__ __device__ constexpr int nst_of(int mode) { return mode == 0 ? HB_NST_DQ : HB_NST_DKV; }
 constexpr int RES_BYTES = BM * HD * 2;        // 32 KB: two 64-column slabs of 128 rows
 constexpr int RES_SLAB = RES_BYTES / 2;
 constexpr int SUBT_BYTES = SUB * HD * 2;      // 16 KB: two 64-column slabs of 64 rows
 constexpr int SUBT_SLAB = SUBT_BYTES / 2;
 constexpr int STAGE_BYTES = 2 * SUBT_BYTES;
-constexpr int THREADS = 384;
-constexpr int SMEM_BYTES = 2 * RES_BYTES + NST * STAGE_BYTES + 1024;
+constexpr int THREADS = 512;  // 8 element-wise warps, 4 single-lane service warps, 4 epilogue warps
+// accumulator buffers: DQ has TMEM for three (its output needs 128 columns), DKV for two
+__host__ __device__ constexpr int nb_of(int mode) { return mode == 0 ? 3 : 2; }
+__host__ __device__ constexpr int smem_bytes_of(int mode) { return 2 * RES_BYTES + nst_of(mode) * STAGE_BYTES + 1024; }
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int MODE_DQ = 0, MODE_DKV = 1;
 
 enum Bar {
-    RES_FULL = 0, OUT_FULL, EPI_DONE, DRAIN,
-    S_FULL,                      // [2] acc1 / acc2 of buffer b written
-    P_READY = S_FULL + 2,        // [2] P / dS of buffer b written, 128 arrivals
-    ST_FULL = P_READY + 2, ST_EMPTY = ST_FULL + NST,
-    NUM_BARS = ST_EMPTY + NST
+    RES_FULL = 0, RES_EMPTY, OUT_FULL, EPI_DONE, DRAIN,
+    S_FULL,                      // [NB] acc1 / acc2 of buffer b written
+    P_READY = S_FULL + 3,        // [NB] P / dS of buffer b written, 256 arrivals
+    ST_FULL = P_READY + 3, ST_EMPTY = ST_FULL + NST_MAX,
+    STAT_FULL = ST_EMPTY + NST_MAX,   // DKV: statistics of the streamed rows of ring slot s written
+    NUM_BARS = STAT_FULL + NST_MAX
 };
 
 struct Params {
@@ -71,6 +84,7 @@ struct Params {
     __nv_bfloat16 *out_b; // DKV: dv
     float scale, scale_log2;
     int S;
+    int out_align32;      // outputs and strides 32-byte aligned: 32-byte stores allowed
     int *status;
 };
 
@@ -92,12 +106,15 @@ __device__ __forceinline__ void issue_rt(uint32_t tmem_acc, uint32_t sR, uint32_
 
 // out (+)= A T: A (128 x 64, bf16) from TMEM, the streamed sub-block row-major in smem
 // (N-major operand: 64 rows of K, two 64-column slabs of N).
+// A sits where each element-wise warpgroup left it: the bf16 pairs of streamed rows
+// [32 w, 32 w + 32) occupy columns [32 w, 32 w + 16) of the fp32 block they were computed from.
 __device__ __forceinline__ void issue_at(uint32_t tmem_out, uint32_t tmem_a, uint32_t sT, bool accumulate) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
     const uint64_t db = smem_desc_sw128(sT, SUBT_SLAB, 1024);
 #pragma unroll
     for (int k = 0; k < SUB / 16; ++k)
-        mma_ts(tmem_out, tmem_a + k * 8, db + (uint64_t)((k * 2048) >> 4), IDESC, (accumulate || k > 0) ? 1u : 0u);
+        mma_ts(tmem_out, tmem_a + (k >> 1) * 32 + (k & 1) * 8, db + (uint64_t)((k * 2048) >> 4), IDESC,
+               (accumulate || k > 0) ? 1u : 0u);
 }
 
 template <int MODE>
@@ -105,16 +122,19 @@ __global__ void __launch_bounds__(THREADS, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant__ CUtensorMap tmR2,
                 const __grid_constant__ CUtensorMap tmT1, const __grid_constant__ CUtensorMap tmT2,
                 const Params prm) {
+    constexpr int NST = nst_of(MODE);
+    constexpr int NB = nb_of(MODE), LA = NB - 1;          // MMAs run LA sub-blocks ahead of the element-wise step
+    constexpr uint32_t OUT_A = MODE == MODE_DKV ? 256 : 384, OUT_B = 384;  // TMEM columns of the outputs
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[NUM_BARS];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ __align__(16) float stats[NST][2][SUB];  // DKV: lse (base 2) and delta of the streamed query rows
+    __shared__ __align__(16) float stats[MODE == MODE_DKV ? NST : 1][2][SUB];  // DKV: lse (base 2), delta of streamed rows
 
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sR1 = smem_u32(smem), sR2 = sR1 + RES_BYTES;
     const uint32_t sST = sR2 + RES_BYTES;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, warp = tid >> 5;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -122,8 +142,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
         abort_flag = 0;
         for (int i = 0; i < NUM_BARS; ++i) {
             uint32_t count = 1;
-            if (i == EPI_DONE) count = 256;
-            if (i >= P_READY && i < P_READY + 2) count = 128;
+            if (i == EPI_DONE) count = 128;
+            if (i >= P_READY && i < P_READY + 3) count = 256;
             mbar_init(bar(i), count);
         }
         mbar_fence_init();
@@ -142,60 +162,23 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     }
     if (warp == 8) {
-        // ------------------------------------------------------------ producer (whole warp)
-        if (lane == 0) {
-            prefetch_tmap(&tmR1);
-            prefetch_tmap(&tmR2);
+        // ------------------------------------------------ producer of the streamed sub-blocks
+        if (elect_one()) {
             prefetch_tmap(&tmT1);
             prefetch_tmap(&tmT2);
-        }
-        uint32_t g = 0, uc = 0;
-        bool ok = true;
-        for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
-            const WorkUnit unit = prm.units[u];
-            const WorkItem wi = prm.work[unit.item];
-            const int bh = unit.bh;
-            const int b = bh / prm.heads, h = bh % prm.heads;
-            if (lane == 0) {
-                // the resident tiles are free once every MMA of the previous unit has retired
-                if (uc > 0) ok = wait_or_abort(bar(OUT_FULL), (uc - 1) & 1, &abort_flag, prm.status, 0x401);
-                if (ok) {
-                    mbar_expect_tx(bar(RES_FULL), 2 * RES_BYTES);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t off = (i >> 1) * RES_SLAB + (i & 1) * (SUB * 128);
-                        tma_load_4d(sR1 + off, &tmR1, bar(RES_FULL), (i >> 1) * 64, wi.q_start + (i & 1) * SUB, h, b);
-                        tma_load_4d(sR2 + off, &tmR2, bar(RES_FULL), (i >> 1) * 64, wi.q_start + (i & 1) * SUB, h, b);
-                    }
-                }
-            }
-            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
-                const int nb = sub_blocks(wi, seg);
-                for (int j = 0; ok && j < nb; ++j, ++g) {
-                    const int row = wi.seg_start[seg] + j * SUB;
-                    const uint32_t s = g % NST, ph = (g / NST) & 1;
-                    if (lane == 0) ok = wait_or_abort(bar(ST_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x402);
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (!ok) break;
-                    if (MODE == MODE_DKV) {
-                        // per-query statistics of the streamed rows; rows beyond the range get
-                        // lse = +inf, which turns their weights into exact zeros
-                        const int valid = min(SUB, wi.seg_len[seg] - j * SUB);
-#pragma unroll
-                        for (int i = 0; i < SUB / 32; ++i) {
-                            const int c = lane + 32 * i;
-                            float l2 = __int_as_float(0x7f800000), dl = 0.f;
-                            if (c < valid) {
-                                l2 = prm.lse[(long long)bh * prm.S + row + c] * 1.4426950408889634f;
-                                dl = prm.delta[(long long)bh * prm.S + row + c];
-                            }
-                            stats[s][0][c] = l2;
-                            stats[s][1][c] = dl;
-                        }
-                        __syncwarp();
-                    }
-                    if (lane == 0) {
+            uint32_t g = 0;
+            bool ok = true;
+            for (int u = u_begin; ok && u < u_end; ++u) {
+                const WorkUnit unit = prm.units[u];
+                const WorkItem wi = prm.work[unit.item];
+                const int b = unit.bh / prm.heads, h = unit.bh % prm.heads;
+                for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
+                    const int nb = sub_blocks(wi, seg);
+                    for (int j = 0; j < nb; ++j, ++g) {
+                        const int row = wi.seg_start[seg] + j * SUB;
+                        const uint32_t s = g % NST, ph = (g / NST) & 1;
+                        ok = wait_or_abort(bar(ST_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x402);
+                        if (!ok) break;
                         const uint32_t dst = sST + s * STAGE_BYTES;
                         mbar_expect_tx(bar(ST_FULL + s), STAGE_BYTES);
                         tma_load_4d(dst, &tmT1, bar(ST_FULL + s), 0, row, h, b);
@@ -205,52 +188,242 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                     }
                 }
             }
-        }
-        if (!ok && lane == 0) {
-            // let every copy already issued land before the CTA retires
-            const long long t0 = clock64();
-            while (clock64() - t0 < 2000000) {
+            if (!ok) {
+                // let every copy already issued land before the CTA retires
+                const long long t0 = clock64();
+                while (clock64() - t0 < 2000000) {
+                }
             }
+        }
+    } else if (warp == 10) {
+        // ------------------------------------------------ loader of the resident tiles
+        // A thread of its own, so that the sub-block producer can run ahead into the next unit
+        // while this one waits for the resident tiles to be released.
+        if (elect_one()) {
+            prefetch_tmap(&tmR1);
+            prefetch_tmap(&tmR2);
+            uint32_t uc = 0;
+            bool ok = true;
+            for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
+                const WorkUnit unit = prm.units[u];
+                const WorkItem wi = prm.work[unit.item];
+                const int b = unit.bh / prm.heads, h = unit.bh % prm.heads;
+                // free once the last R T^T MMA of the previous unit has retired
+                if (uc > 0) ok = wait_or_abort(bar(RES_EMPTY), (uc - 1) & 1, &abort_flag, prm.status, 0x401);
+                if (!ok) break;
+                mbar_expect_tx(bar(RES_FULL), 2 * RES_BYTES);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t off = (i >> 1) * RES_SLAB + (i & 1) * (SUB * 128);
+                    tma_load_4d(sR1 + off, &tmR1, bar(RES_FULL), (i >> 1) * 64, wi.q_start + (i & 1) * SUB, h, b);
+                    tma_load_4d(sR2 + off, &tmR2, bar(RES_FULL), (i >> 1) * 64, wi.q_start + (i & 1) * SUB, h, b);
+                }
+                if (u + 1 < u_end) {
+                    // pull the next unit's resident tiles into L2 while this unit runs
+                    const WorkUnit nu = prm.units[u + 1];
+                    const int nq = prm.work[nu.item].q_start;
+                    const int nb_ = nu.bh / prm.heads, nh = nu.bh % prm.heads;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        tma_prefetch_4d(&tmR1, (i >> 1) * 64, nq + (i & 1) * SUB, nh, nb_);
+                        tma_prefetch_4d(&tmR2, (i >> 1) * 64, nq + (i & 1) * SUB, nh, nb_);
+                    }
+                }
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < 2000000) {
+                }
+            }
+        }
+    } else if (warp == 11) {
+        // ------------------------------------------------ DKV: statistics of the streamed query rows
+        // lse (base 2) and delta of the 64 rows of every sub-block go to shared memory, two
+        // sub-blocks ahead of use; rows beyond the range get lse = +inf, which turns their
+        // weights into exact zeros.
+        if (MODE == MODE_DKV) {
+            const int lane = tid & 31;
+            struct It {
+                int u, seg, j, bh;
+                WorkItem wi;
+                bool valid;
+            };
+            auto load_unit = [&](It &it) {
+                it.valid = it.u < u_end;
+                if (it.valid) {
+                    const WorkUnit unit = prm.units[it.u];
+                    it.wi = prm.work[unit.item];
+                    it.bh = unit.bh;
+                }
+            };
+            auto advance = [&](It &it) {
+                if (++it.j >= sub_blocks(it.wi, it.seg)) {
+                    it.j = 0;
+                    if (++it.seg >= it.wi.n_seg) {
+                        it.seg = 0;
+                        ++it.u;
+                        load_unit(it);
+                    }
+                }
+            };
+            auto fetch = [&](const It &it, float (&l2)[2], float (&dl)[2]) {
+                if (!it.valid) return;
+                const int row = it.wi.seg_start[it.seg] + it.j * SUB;
+                const int valid = min(SUB, it.wi.seg_len[it.seg] - it.j * SUB);
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int c = lane + 32 * i;
+                    l2[i] = __int_as_float(0x7f800000);
+                    dl[i] = 0.f;
+                    if (c < valid) {
+                        l2[i] = __ldg(prm.lse + (long long)it.bh * prm.S + row + c) * 1.4426950408889634f;
+                        dl[i] = __ldg(prm.delta + (long long)it.bh * prm.S + row + c);
+                    }
+                }
+            };
+            uint32_t g = 0;
+            bool ok = true;
+            auto publish = [&](const float (&l2)[2], const float (&dl)[2]) {
+                const uint32_t s = g % NST, ph = (g / NST) & 1;
+                if (lane == 0) ok = wait_or_abort(bar(ST_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x701);
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) return;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    stats[s][0][lane + 32 * i] = l2[i];
+                    stats[s][1][lane + 32 * i] = dl[i];
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(STAT_FULL + s));
+                ++g;
+            };
+            It cur{u_begin, 0, 0, 0, WorkItem{}, false}, pre{u_begin, 0, 0, 0, WorkItem{}, false};
+            load_unit(cur);
+            load_unit(pre);
+            float al2[2], adl[2], bl2[2], bdl[2];
+            fetch(pre, al2, adl);
+            if (pre.valid) advance(pre);
+            fetch(pre, bl2, bdl);
+            if (pre.valid) advance(pre);
+            while (ok && cur.valid) {
+                publish(al2, adl);
+                if (!ok) break;
+                advance(cur);
+                fetch(pre, al2, adl);
+                if (pre.valid) advance(pre);
+                if (!cur.valid) break;
+                publish(bl2, bdl);
+                if (!ok) break;
+                advance(cur);
+                fetch(pre, bl2, bdl);
+                if (pre.valid) advance(pre);
+            }
+        }
+    } else if (warp >= 12) {
+        // ------------------------------------------------ epilogue: accumulators -> bf16 -> global
+        // Its own warpgroup, so that the element-wise warps move on to the next unit at once.
+        const int r = tid & 127;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        uint32_t uc = 0;
+        bool ok = true;
+        for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
+            const WorkUnit unit = prm.units[u];
+            const WorkItem wi = prm.work[unit.item];
+            const int b = unit.bh / prm.heads, h = unit.bh % prm.heads;
+            const bool row_ok = r < wi.q_rows;
+            ok = wait_or_abort(bar(OUT_FULL), uc & 1, &abort_flag, prm.status, 0x605);
+            if (!ok) break;
+            tc_fence_after();
+            const long long roff = (long long)b * prm.stride_b + (long long)h * prm.stride_h +
+                                   (long long)(wi.q_start + r) * prm.stride_s;
+            constexpr int NCH = (MODE == MODE_DKV) ? 8 : 4;   // DKV: dK then dV
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem + lane_addr + OUT_A + c * 32, o);
+                tmem_wait_ld();
+                if (row_ok) {
+                    __nv_bfloat16 *orow = (c >= 4 ? prm.out_b : prm.out_a) + roff + (c & 3) * 32;
+                    const float mul = c >= 4 ? 1.f : prm.scale;
+                    uint32_t w[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        w[i] = pack_bf16(__uint_as_float(o[2 * i]) * mul, __uint_as_float(o[2 * i + 1]) * mul);
+                    if (prm.out_align32) {
+                        st_global_v8(orow, w);
+                        st_global_v8(orow + 16, w + 8);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)
+                            *reinterpret_cast<uint4 *>(orow + 2 * i) = make_uint4(w[i], w[i + 1], w[i + 2], w[i + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(EPI_DONE));
         }
     } else if (warp == 9) {
         // ---------------------------------------------------------- MMA issuer
         if (elect_one()) {
             uint32_t g = 0, uc = 0;
-            uint32_t cP[2] = {0, 0};
+            uint32_t cP[3] = {0, 0, 0};
             bool ok = true;
+#ifdef HB_BWD_TIMING
+            long long tw_res = 0, tw_st = 0, tw_epi = 0, tw_p = 0, tw_st0 = 0, tw_p0 = 0, t_mark, t_start = clock64();
+#define TMARK() t_mark = clock64()
+#define TACC(x) x += clock64() - t_mark
+#else
+#define TMARK()
+#define TACC(x)
+#endif
             for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
                 const WorkItem wi = prm.work[prm.units[u].item];
                 const int n = wi.kv_blocks;  // sub-blocks of this item
+                TMARK();
                 ok = wait_or_abort(bar(RES_FULL), uc & 1, &abort_flag, prm.status, 0x501);
+                TACC(tw_res);
                 if (!ok) break;
-                for (int s = 0; s <= n; ++s) {
+                for (int s = 0; s < n + LA; ++s) {
                     if (s < n) {
                         const uint32_t e = g + s, slot = e % NST;
+                        TMARK();
                         ok = wait_or_abort(bar(ST_FULL + slot), (e / NST) & 1, &abort_flag, prm.status, 0x502);
+                        TACC(tw_st);
+#ifdef HB_BWD_TIMING
+                        if (s < 2) tw_st0 += clock64() - t_mark;
+#endif
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t sT = sST + slot * STAGE_BYTES;
-                        const uint32_t acc = tmem + (s & 1) * 128;
+                        const uint32_t acc = tmem + (s % NB) * 128;
                         issue_rt(acc, sR1, sT);
                         issue_rt(acc + 64, sR2, sT + SUBT_BYTES);
-                        mma_commit(bar(S_FULL + (s & 1)));
+                        mma_commit(bar(S_FULL + (s % NB)));
+                        if (s == n - 1) mma_commit(bar(RES_EMPTY));
                     }
-                    if (s >= 1) {
-                        const int sp = s - 1, bf = sp & 1;
+                    if (s >= LA) {
+                        const int sp = s - LA, bf = sp % NB;
                         const uint32_t e = g + sp, slot = e % NST;
                         if (sp == 0 && uc > 0) {
                             // the previous unit's accumulators have been read out
+                            TMARK();
                             ok = wait_or_abort(bar(EPI_DONE), (uc - 1) & 1, &abort_flag, prm.status, 0x503);
+                            TACC(tw_epi);
                             if (!ok) break;
                         }
+                        TMARK();
                         ok = wait_or_abort(bar(P_READY + bf), cP[bf] & 1, &abort_flag, prm.status, 0x504 + bf);
+                        TACC(tw_p);
+#ifdef HB_BWD_TIMING
+                        if (sp < 2) tw_p0 += clock64() - t_mark;
+#endif
                         if (!ok) break;
                         ++cP[bf];
                         tc_fence_after();
                         const uint32_t sT = sST + slot * STAGE_BYTES;
                         const uint32_t acc = tmem + bf * 128;
-                        issue_at(tmem + 256, acc + 64, sT, sp > 0);                         // dS   x T1
-                        if (MODE == MODE_DKV) issue_at(tmem + 384, acc, sT + SUBT_BYTES, sp > 0);  // P^T x T2
+                        issue_at(tmem + OUT_A, acc + 64, sT, sp > 0);                                  // dS  x T1
+                        if (MODE == MODE_DKV) issue_at(tmem + OUT_B, acc, sT + SUBT_BYTES, sp > 0);  // P^T x T2
                         mma_commit(bar(ST_EMPTY + slot));
                     }
                 }
@@ -261,16 +434,25 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
             // every MMA issued above has retired before TMEM is released
             mma_commit(bar(DRAIN));
             wait_or_abort(bar(DRAIN), 0, &abort_flag, prm.status, 0x507);
+#ifdef HB_BWD_TIMING
+            atomicAdd(prm.status + 32 + MODE * 8 + 0, (int)(tw_res >> 6));
+            atomicAdd(prm.status + 32 + MODE * 8 + 1, (int)(tw_st >> 6));
+            atomicAdd(prm.status + 32 + MODE * 8 + 2, (int)(tw_epi >> 6));
+            atomicAdd(prm.status + 32 + MODE * 8 + 3, (int)(tw_p >> 6));
+            atomicAdd(prm.status + 32 + MODE * 8 + 4, (int)((clock64() - t_start) >> 6));
+            atomicMax(prm.status + 32 + MODE * 8 + 5, (int)((clock64() - t_start) >> 6));
+            atomicAdd(prm.status + 32 + MODE * 8 + 6, (int)(tw_st0 >> 6));
+            atomicAdd(prm.status + 32 + MODE * 8 + 7, (int)(tw_p0 >> 6));
+#endif
         }
     } else if (warp < 8) {
         // ------------------------------------ element-wise step + epilogue, warpgroup wg
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
         const int wg = warp >> 2;
         const int r = tid & 127;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tAcc = tmem + lane_addr + wg * 128;
         const float scale_log2 = prm.scale_log2;
-        uint32_t cS = 0, g = 0, uc = 0;
+        uint32_t cS[3] = {0, 0, 0}, g = 0, uc = 0;
         bool ok = true;
         for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
             const WorkUnit unit = prm.units[u];
@@ -288,93 +470,59 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                 const int nb = sub_blocks(wi, seg);
                 for (int j = 0; j < nb; ++j, ++s) {
-                    if ((s & 1) != wg) continue;
-                    const int valid = min(SUB, wi.seg_len[seg] - j * SUB);
+                    const int bf = s % NB;
+                    // this warpgroup's 32 columns of the sub-block
+                    const int valid = min(SUB, wi.seg_len[seg] - j * SUB) - wg * 32;
+                    const uint32_t tAcc = tmem + lane_addr + bf * 128;
                     const uint32_t e = g + s, slot = e % NST;
                     if (MODE == MODE_DKV) {
-                        // the statistics were written before the producer's arrival on this barrier
-                        ok = wait_or_abort(bar(ST_FULL + slot), (e / NST) & 1, &abort_flag, prm.status, 0x601 + wg);
+                        ok = wait_or_abort(bar(STAT_FULL + slot), (e / NST) & 1, &abort_flag, prm.status, 0x601 + wg);
                         if (!ok) break;
                     }
-                    ok = wait_or_abort(bar(S_FULL + wg), cS & 1, &abort_flag, prm.status, 0x603 + wg);
+                    ok = wait_or_abort(bar(S_FULL + bf), cS[bf] & 1, &abort_flag, prm.status, 0x603 + wg);
                     if (!ok) break;
-                    ++cS;
                     tc_fence_after();
-                    uint32_t a1[SUB], a2[SUB];
-                    tmem_ld32(tAcc, *reinterpret_cast<uint32_t(*)[32]>(&a1[0]));
-                    tmem_ld32(tAcc + 32, *reinterpret_cast<uint32_t(*)[32]>(&a1[32]));
-                    tmem_ld32(tAcc + 64, *reinterpret_cast<uint32_t(*)[32]>(&a2[0]));
-                    tmem_ld32(tAcc + 96, *reinterpret_cast<uint32_t(*)[32]>(&a2[32]));
+                    uint32_t a1[32], a2[32];
+                    tmem_ld32(tAcc + wg * 32, a1);
+                    tmem_ld32(tAcc + 64 + wg * 32, a2);
                     tmem_wait_ld();
+                    uint32_t pk[16], dk[16];
 #pragma unroll
-                    for (int c = 0; c < SUB / 32; ++c) {
-                        uint32_t pk[16], dk[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int c0 = c * 32 + 2 * i;
-                            float l0, l1, d0, d1;
-                            if (MODE == MODE_DKV) {
-                                const float2 l2 = *reinterpret_cast<const float2 *>(&stats[slot][0][c0]);
-                                const float2 dl = *reinterpret_cast<const float2 *>(&stats[slot][1][c0]);
-                                l0 = l2.x; l1 = l2.y; d0 = dl.x; d1 = dl.y;
-                            } else {
-                                l0 = l1 = row_l2;
-                                d0 = d1 = row_dl;
-                            }
-                            float p0 = ex2(fmaf(__uint_as_float(a1[c0]), scale_log2, -l0));
-                            float p1 = ex2(fmaf(__uint_as_float(a1[c0 + 1]), scale_log2, -l1));
-                            if (MODE == MODE_DQ) {
-                                // keys beyond the end of the range
-                                if (c0 >= valid) p0 = 0.f;
-                                if (c0 + 1 >= valid) p1 = 0.f;
-                            }
-                            const float s0 = p0 * (__uint_as_float(a2[c0]) - d0);
-                            const float s1 = p1 * (__uint_as_float(a2[c0 + 1]) - d1);
-                            pk[i] = pack_bf16(p0, p1);
-                            dk[i] = pack_bf16(s0, s1);
+                    for (int i = 0; i < 16; ++i) {
+                        const int c0 = 2 * i;
+                        float l0, l1, d0, d1;
+                        if (MODE == MODE_DKV) {
+                            const float2 l2 = *reinterpret_cast<const float2 *>(&stats[slot][0][wg * 32 + c0]);
+                            const float2 dl = *reinterpret_cast<const float2 *>(&stats[slot][1][wg * 32 + c0]);
+                            l0 = l2.x; l1 = l2.y; d0 = dl.x; d1 = dl.y;
+                        } else {
+                            l0 = l1 = row_l2;
+                            d0 = d1 = row_dl;
                         }
-                        if (MODE == MODE_DKV) tmem_st16(tAcc + c * 16, pk);
-                        tmem_st16(tAcc + 64 + c * 16, dk);
+                        float p0 = ex2(fmaf(__uint_as_float(a1[c0]), scale_log2, -l0));
+                        float p1 = ex2(fmaf(__uint_as_float(a1[c0 + 1]), scale_log2, -l1));
+                        if (MODE == MODE_DQ) {
+                            // keys beyond the end of the range
+                            if (c0 >= valid) p0 = 0.f;
+                            if (c0 + 1 >= valid) p1 = 0.f;
+                        }
+                        const float s0 = p0 * (__uint_as_float(a2[c0]) - d0);
+                        const float s1 = p1 * (__uint_as_float(a2[c0 + 1]) - d1);
+                        pk[i] = pack_bf16(p0, p1);
+                        dk[i] = pack_bf16(s0, s1);
                     }
+                    // in place: the bf16 pairs land in the first half of the 32 fp32 columns this
+                    // warpgroup has just read, so no other thread's data is touched
+                    if (MODE == MODE_DKV) tmem_st16(tAcc + wg * 32, pk);
+                    tmem_st16(tAcc + 64 + wg * 32, dk);
+                    ++cS[bf];
                     tmem_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar(P_READY + wg));
+                    mbar_arrive(bar(P_READY + bf));
                 }
             }
             if (!ok) break;
             g += wi.kv_blocks;
-            // epilogue: accumulators -> bf16 -> global; rows beyond the item are dropped
-            ok = wait_or_abort(bar(OUT_FULL), uc & 1, &abort_flag, prm.status, 0x605 + wg);
-            if (!ok) break;
-            tc_fence_after();
-            {
-                // DQ: warpgroup wg stores columns [64 wg, +64) of dQ; DKV: wg 0 stores dK, wg 1 stores dV
-                const uint32_t tOut = tmem + lane_addr + 256 + (MODE == MODE_DKV ? wg * 128 : wg * 64);
-                __nv_bfloat16 *base = (MODE == MODE_DKV && wg == 1) ? prm.out_b : prm.out_a;
-                __nv_bfloat16 *orow = base + (long long)b * prm.stride_b + (long long)h * prm.stride_h +
-                                      (long long)(wi.q_start + r) * prm.stride_s + (MODE == MODE_DKV ? 0 : wg * 64);
-                const float mul = (MODE == MODE_DKV && wg == 1) ? 1.f : prm.scale;
-                constexpr int NCH = (MODE == MODE_DKV) ? 4 : 2;
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tOut + c * 32, o);
-                    tmem_wait_ld();
-                    if (row_ok) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(o[i]) * mul, __uint_as_float(o[i + 1]) * mul);
-                            w.y = pack_bf16(__uint_as_float(o[i + 2]) * mul, __uint_as_float(o[i + 3]) * mul);
-                            w.z = pack_bf16(__uint_as_float(o[i + 4]) * mul, __uint_as_float(o[i + 5]) * mul);
-                            w.w = pack_bf16(__uint_as_float(o[i + 6]) * mul, __uint_as_float(o[i + 7]) * mul);
-                            *reinterpret_cast<uint4 *>(orow + c * 32 + i) = w;
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(bar(EPI_DONE));
         }
     }
 
@@ -494,10 +642,10 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_of(MODE_DQ));
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            SMEM_BYTES);
+                                            smem_bytes_of(MODE_DKV));
     });
     HB_CUDA(attr_err);
     return HILBERTA_OK;
@@ -532,13 +680,15 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.S = p->S;
     prm.status = p->d_status;
+    prm.out_align32 = ((((uintptr_t)dq | (uintptr_t)dk | (uintptr_t)dv) & 31) == 0 &&
+                       ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
     prm.out_a = (__nv_bfloat16 *)dq;
     prm.out_b = nullptr;
-    attn_bwd_kernel<MODE_DQ><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mq, mdo, mk, mv, prm);
+    attn_bwd_kernel<MODE_DQ><<<p->n_bwd_cta, THREADS, smem_bytes_of(MODE_DQ), stream>>>(mq, mdo, mk, mv, prm);
     HB_LAUNCHED();
     prm.out_a = (__nv_bfloat16 *)dk;
     prm.out_b = (__nv_bfloat16 *)dv;
-    attn_bwd_kernel<MODE_DKV><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mk, mv, mq, mdo, prm);
+    attn_bwd_kernel<MODE_DKV><<<p->n_bwd_cta, THREADS, smem_bytes_of(MODE_DKV), stream>>>(mk, mv, mq, mdo, prm);
     HB_LAUNCHED();
     return HILBERTA_OK;
 }
