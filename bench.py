@@ -202,6 +202,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the dense / SDPA context rows")
+    ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass row")
     ap.add_argument("--schedule", action="store_true",
                     help="also time the 57-layer per-step schedule (one permute, 57 forwards with the "
                          "per-layer offsets, one unpermute) on the chosen workload's shape")
@@ -378,6 +379,42 @@ def main():
         context_rows["sparse_speedup_vs_dense_this_build"] = (
             context_rows["dense_this_build"]["ms"] / fwd_avg if "ms" in context_rows["dense_this_build"] else None)
 
+    # ---- backward pass (not part of the metric): dq, dk, dv on the same plan and inputs
+    backward = None
+    if world == 1 and not args.no_backward and wl.dtype == "bf16":
+        lse = torch.empty((wl.batch, wl.heads, wl.S), device="cuda", dtype=torch.float32)
+        g = torch.Generator().manual_seed(wl.seed + 7)
+        dop = torch.randn(qp.shape, generator=g).to(torch.bfloat16).cuda()
+        grads = [torch.empty_like(qp) for _ in range(3)]
+        plan.forward_lse(qp, kp, vp, op, lse)
+        for _ in range(3):
+            plan.backward(dop, qp, kp, vp, op, lse, *grads)
+        torch.cuda.synchronize()
+        n_b = max(5, min(args.steps, 30))
+        bev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_b)]
+        l0 = hb.launch_count()
+        for a, b_ in bev:
+            a.record(stream)
+            plan.backward(dop, qp, kp, vp, op, lse, *grads)
+            b_.record(stream)
+        torch.cuda.synchronize()
+        assert plan.status() == 0, "device-side wait timed out"
+        assert all(torch.isfinite(t.float()).all() for t in grads)
+        bms = sorted(a.elapsed_time(b_) for a, b_ in bev)
+        b_med = bms[len(bms) // 2]
+        bflops = 2.5 * flops          # five contractions of 2 D flops per kept pair
+        backward = {
+            "ms_per_call_median": b_med, "ms_per_call_min": bms[0],
+            "useful_tflops": bflops / (b_med * 1e-3) / 1e12,
+            "useful_gflop_per_call": bflops / 1e9,
+            "executed_tflops": 1.4 * bflops / (b_med * 1e-3) / 1e12,
+            "frac_of_measured_burst_peak": bflops / (b_med * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "launches_per_call": (hb.launch_count() - l0) // n_b,
+            "note": "useful = 10 D flops per kept pair (dS, dQ, dK, dV and the recomputed scores); executed = 14 D: "
+                    "the dQ and the dK/dV kernels each recompute the scores and dP",
+        }
+        del dop, grads, lse
+
     schedule = None
     if args.schedule:
         from paper_2509_26538_b200.inputs import SCHEDULE_LAYERS, schedule_offset
@@ -442,7 +479,7 @@ def main():
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_source": peaks["source"] + " burst",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "traffic": FORWARD_DRAM_TRAFFIC_BYTES.get(wl.name)},
-        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "schedule57": schedule,
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "backward": backward, "schedule57": schedule,
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
                              "(4.36 ms per call at 2048^2, 16 tiles)", "same_gpu": context_rows},
     }
