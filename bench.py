@@ -379,6 +379,31 @@ def main():
         context_rows["sparse_speedup_vs_dense_this_build"] = (
             context_rows["dense_this_build"]["ms"] / fwd_avg if "ms" in context_rows["dense_this_build"] else None)
 
+    # ---- the whole step as ONE launch: entry and exit gathers fused into the attention kernel
+    fused = None
+    if world == 1:
+        of = torch.empty_like(qd)
+        for _ in range(3):
+            plan.forward_fused(qd, kd, vd, of, True, True)
+        torch.cuda.synchronize()
+        n_f = max(5, min(args.steps, 30))
+        fev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_f)]
+        for a, b_ in fev:
+            a.record(stream)
+            plan.forward_fused(qd, kd, vd, of, True, True)
+            b_.record(stream)
+        torch.cuda.synchronize()
+        assert plan.status() == 0, "device-side wait timed out"
+        view = torch.int16 if wl.dtype == "bf16" else torch.int32
+        assert torch.equal(of.view(view), od.view(view)), "fused step differs from permute + forward + unpermute"
+        fms = sorted(a.elapsed_time(b_) for a, b_ in fev)
+        f_med = fms[len(fms) // 2]
+        fused = {"ms_per_step_median": f_med, "ms_per_step_min": fms[0],
+                 "useful_tflops": flops / (f_med * 1e-3) / 1e12,
+                 "api": "hilberta_forward_fused(in_original=1, out_original=1): q, k, v and out in ORIGINAL order, "
+                        "one launch, no permuted copies; bit-identical to the step above"}
+        del of
+
     # ---- backward pass (not part of the metric): dq, dk, dv on the same plan and inputs
     backward = None
     if world == 1 and not args.no_backward and wl.dtype == "bf16":
@@ -479,7 +504,7 @@ def main():
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_source": peaks["source"] + " burst",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "traffic": FORWARD_DRAM_TRAFFIC_BYTES.get(wl.name)},
-        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "backward": backward, "schedule57": schedule,
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "fused_step": fused, "backward": backward, "schedule57": schedule,
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
                              "(4.36 ms per call at 2048^2, 16 tiles)", "same_gpu": context_rows},
     }

@@ -248,6 +248,19 @@ int hilberta_permute(const void *src, void *dst, const hilberta_plan_t *plan, in
 int hilberta_unpermute(const void *src, void *dst, const hilberta_plan_t *plan, int batch,
                        int row_elems, int dtype, void *stream);
 
+/* The attention launch with the entry and / or exit gather of Sec. 3.4 fused in,
+ * for the first and last attention layer of a step (or a single layer):
+ *   in_original  != 0 : q, k, v are in ORIGINAL token order; every tile row is read
+ *                       through the permutation (physical row p from row
+ *                       phys2orig[p]) on its way into shared memory, so no permuted
+ *                       copy of q, k, v is ever written;
+ *   out_original != 0 : `out` is written in ORIGINAL order (as
+ *                       hilberta_forward_unpermute does).
+ * With both flags zero this is hilberta_forward.  Same shapes, strides, alignment,
+ * stream and error rules as hilberta_forward; bf16 and fp32 bindings. */
+int hilberta_forward_fused(const void *q, const void *k, const void *v, void *out,
+                           const hilberta_plan_t *plan, int in_original, int out_original, void *stream);
+
 /* Host-buffer form of the whole path, for callers that hold activations in host
  * memory: copies q, k, v (HOST pointers, ORIGINAL order, dense
  * [batch, heads, S, head_dim]) to the device, permutes them, runs the forward,

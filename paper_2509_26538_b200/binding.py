@@ -25,7 +25,8 @@ BF16, FP32 = 0, 1
 SYMBOLS = (
     "hilberta_plan", "hilberta_plan_groups", "hilberta_plan_destroy", "hilberta_plan_export",
     "hilberta_plan_bind",
-    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_lse", "hilberta_backward",
+    "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_fused", "hilberta_forward_lse",
+    "hilberta_backward",
     "hilberta_backward_static", "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
@@ -70,6 +71,8 @@ def lib():
     L.hilberta_forward.restype = i32
     L.hilberta_forward_unpermute.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_unpermute.restype = i32
+    L.hilberta_forward_fused.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
+    L.hilberta_forward_fused.restype = i32
     L.hilberta_forward_lse.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.hilberta_forward_lse.restype = i32
     L.hilberta_backward.argtypes = [vp] * 11
@@ -192,6 +195,13 @@ class Plan:
         """Forward whose output lands in ORIGINAL token order (exit gather fused in)."""
         _check(lib().hilberta_forward_unpermute(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                                 self._h, _stream_ptr(stream)), "hilberta_forward_unpermute")
+        return out
+
+    def forward_fused(self, q, k, v, out, in_original=True, out_original=True, stream=None):
+        """Forward with the entry gather (q, k, v in ORIGINAL order) and / or the exit gather fused in."""
+        _check(lib().hilberta_forward_fused(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), self._h,
+                                            int(bool(in_original)), int(bool(out_original)), _stream_ptr(stream)),
+               "hilberta_forward_fused")
         return out
 
     def forward_lse(self, q, k, v, out, lse, stream=None):

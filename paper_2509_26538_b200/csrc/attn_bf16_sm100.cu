@@ -85,6 +85,17 @@ struct Params {
     int *status;
 };
 
+// Entry gather fused in (GATHER kernels): q, k, v are in ORIGINAL order and physical row p is read
+// from row in_map[p].  Only the gathering kernel's parameter block carries these fields: growing the
+// plain kernel's block changes its register allocation and costs it 1.5 %.
+template <bool GATHER>
+struct KernelParams : Params {};
+template <>
+struct KernelParams<true> : Params {
+    const int *in_map;
+    const __nv_bfloat16 *gq, *gk, *gv;
+};
+
 __device__ __forceinline__ int item_blocks(const WorkItem &it, int seg) {
     return (it.seg_len[seg] + BN - 1) / BN;
 }
@@ -139,9 +150,20 @@ __device__ __forceinline__ void issue_pv_half(uint32_t tmem_o, uint32_t tmem_p, 
     }
 }
 
+constexpr int GATHER_THREADS = 64;  // warps 10 and 11
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
+// GATHER = false: Q / K / V tiles arrive by TMA from tensors in physical order.
+// GATHER = true : the tensors are in ORIGINAL order (the entry gather of Sec. 3.4 fused in): two loader
+// warps fetch every tile row through the permutation table with 16-byte cp.async copies and place it
+// where a 128-byte-swizzled TMA box would have put it, so everything downstream is unchanged.
+template <bool GATHER>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const Params prm) {
+                 const __grid_constant__ CUtensorMap tmV, const KernelParams<GATHER> prm) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[NUM_BARS];
     __shared__ uint32_t tmem_slot;
@@ -157,7 +179,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < NUM_BARS; ++i)
-            mbar_init(bar(i), (i >= P_READY && i < P_READY + 2 * QT) ? (HB_WARP_ARRIVE ? 4 : 128) : 1);
+        {
+            uint32_t count = 1;
+            if (i >= P_READY && i < P_READY + 2 * QT) count = HB_WARP_ARRIVE ? 4 : 128;
+            if (GATHER && (i == Q_FULL || (i >= KV_FULL && i < KV_FULL + NSTAGE))) count = GATHER_THREADS;
+            mbar_init(bar(i), count);
+        }
         mbar_fence_init();
     }
     if (warp == 8) {
@@ -176,7 +203,90 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     }
-    if (warp == 8) {
+    if constexpr (GATHER) {
+    if (warp == 10 || warp == 11) {
+        // ------------------------------------------------- gathering loaders (entry permute fused in)
+        const int lt = tid - 10 * 32;        // 0 .. 63
+        const int chunk = lt & 15;           // 16-byte piece of a 256-byte row
+        uint32_t kvc = 0, qc = 0;
+        bool ok = true;
+        // The stage's barrier counts one arrival per loader thread; each arrival fires by itself
+        // when that thread's copies into the stage have landed, so the loaders never wait for data.
+        auto publish = [&](uint32_t b) {
+            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(b) : "memory");
+        };
+        // Warp w of the two copies rows [64 w, 64 w + 64) of a tile, two adjacent rows per
+        // instruction (lanes 0-15 one row, lanes 16-31 the next; 16 bytes per lane).  Lane L fetches
+        // the table entries of rows L and 32 + L of that range once per tile; the lanes that copy a
+        // row pick its entry up by shuffle, so the table costs one load latency per tile.
+        const int lane = tid & 31, half = lane >> 4, wrow = (warp - 10) * 64;
+        const uint32_t dst_lane = (uint32_t)((chunk >> 3) * SLAB_BYTES + (wrow + half) * 128);
+        const int c7 = (chunk & 7) ^ half;   // row & 7 = (2 i + half) & 7 = (2 i & 7) ^ half
+        auto load_rows = [&](int row0, int &ia, int &ib) {
+            const int pa = row0 + wrow + lane, pb = pa + 32;
+            ia = pa < prm.S ? __ldg(prm.in_map + pa) : -1;   // rows beyond the sequence are
+            ib = pb < prm.S ? __ldg(prm.in_map + pb) : -1;   // zero-filled, as TMA does
+        };
+        auto copy_tile = [&](uint32_t dst_tile, const __nv_bfloat16 *base, int ia, int ib) {
+            const __nv_bfloat16 *src0 = base + chunk * 8;
+            const uint32_t dst0 = dst_tile + dst_lane;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int orow = __shfl_sync(0xffffffffu, i < 16 ? ia : ib, ((2 * i) & 31) + half);
+                const uint32_t dst = dst0 + i * 256 + ((c7 ^ ((2 * i) & 7)) << 4);
+                cp_async16(dst, src0 + (long long)max(orow, 0) * prm.stride_s, orow >= 0 ? 16 : 0);
+            }
+        };
+        for (int u = u_begin; ok && u < u_end; ++u) {
+            const WorkUnit unit = prm.units[u];
+            const WorkItem wi = prm.work[unit.item];
+            const long long bh_off = (long long)(unit.bh / prm.heads) * prm.stride_b +
+                                     (long long)(unit.bh % prm.heads) * prm.stride_h;
+            const int nt = wi.q_rows > BM ? 2 : 1;
+            ok = wait_or_abort(bar(Q_EMPTY), (qc & 1) ^ 1, &abort_flag, prm.status, 0x111);
+            if (!ok) break;
+            ++qc;
+            for (int t = 0; t < nt; ++t) {
+                int ia, ib;
+                load_rows(wi.q_start + t * BM, ia, ib);
+                copy_tile(sQ + t * TILE_BYTES, prm.gq + bh_off, ia, ib);
+            }
+            publish(bar(Q_FULL));
+            for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
+                const int nb = item_blocks(wi, seg);
+                for (int j = 0; ok && j < nb; ++j) {
+                    // the K and the V tile of a block share their rows; the table entries are
+                    // requested before the wait for a free slot
+                    int ia, ib;
+                    load_rows(wi.seg_start[seg] + j * BN, ia, ib);
+                    for (int kv = 0; kv < 2; ++kv, ++kvc) {
+                        const uint32_t s = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
+#ifdef HB_TIMING
+                        const long long tg0 = clock64();
+#endif
+                        ok = wait_or_abort(bar(KV_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x112);
+                        if (!ok) break;
+#ifdef HB_TIMING
+                        const long long tg1 = clock64();
+#endif
+                        copy_tile(sKV + s * TILE_BYTES, (kv ? prm.gv : prm.gk) + bh_off, ia, ib);
+                        publish(bar(KV_FULL + s));
+#ifdef HB_TIMING
+                        if (lt == 0) {
+                            atomicAdd(prm.status + 24, (int)((tg1 - tg0) >> 4));
+                            atomicAdd(prm.status + 25, (int)((clock64() - tg1) >> 4));
+                            atomicAdd(prm.status + 26, 1);
+                        }
+#endif
+                    }
+                }
+            }
+        }
+        // every copy lands before the CTA retires
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    }
+    }
+    if (!GATHER && warp == 8) {
         // ------------------------------------------------------------ producer
         if (elect_one()) {
             prefetch_tmap(&tmQ);
@@ -242,9 +352,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 ok = wait_or_abort(bar(Q_FULL), qc & 1, &abort_flag, prm.status, 0x201);
                 if (!ok) break;
                 ++qc;
+                // tiles written by cp.async (generic proxy) are read by the tensor core (async proxy)
+                if (GATHER) fence_proxy_async_smem();
                 // S_t(0)
                 ok = wait_or_abort(bar(KV_FULL + slot_of(2 * g)), phase_of(2 * g), &abort_flag, prm.status, 0x202);
                 if (!ok) break;
+                if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t) {
                     issue_qk(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
@@ -264,6 +377,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     }
                     ok = wait_or_abort(bar(KV_FULL + slot_of(eV)), phase_of(eV), &abort_flag, prm.status, 0x204);
                     if (!ok) break;
+                    if (GATHER) fence_proxy_async_smem();
 #ifdef HB_TIMING
                     tm_kv += clock64() - tk0;
 #endif
@@ -650,14 +764,17 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            SMEM_BYTES);
     });
     HB_CUDA(attr_err);
     return HILBERTA_OK;
 }
 
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, cudaStream_t stream) {
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream) {
     if (p->n_work == 0) return HILBERTA_OK;
     CUtensorMap mq, mk, mv;
     int rc;
@@ -679,7 +796,19 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     prm.lse = lse;
     prm.S = p->S;
     prm.out_align32 = (((uintptr_t)out & 31) == 0 && ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
-    attn_bf16_kernel<<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, prm);
+    if (in_map) {
+        KernelParams<true> gprm;
+        static_cast<Params &>(gprm) = prm;
+        gprm.in_map = in_map;
+        gprm.gq = (const __nv_bfloat16 *)q;
+        gprm.gk = (const __nv_bfloat16 *)k;
+        gprm.gv = (const __nv_bfloat16 *)v;
+        attn_bf16_kernel<true><<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, gprm);
+    } else {
+        KernelParams<false> pprm;
+        static_cast<Params &>(pprm) = prm;
+        attn_bf16_kernel<false><<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, pprm);
+    }
     HB_LAUNCHED();
     return HILBERTA_OK;
 }

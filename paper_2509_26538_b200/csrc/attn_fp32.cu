@@ -17,15 +17,16 @@ __global__ void __launch_bounds__(kRowsPerBlock * 32)
 attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
                  float *__restrict__ out, long long stride_b, long long stride_h, long long stride_s,
                  int heads, int S, int P, const int *__restrict__ row_window,
-                 const Window *__restrict__ windows, const int *__restrict__ out_map, float *__restrict__ lse,
-                 float scale) {
+                 const Window *__restrict__ windows, const int *__restrict__ out_map,
+                 const int *__restrict__ in_map, float *__restrict__ lse, float scale) {
     __shared__ float sq[kRowsPerBlock][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * kRowsPerBlock + warp;
     if (row >= S) return;  // whole warp leaves together; no block-wide barrier below
     const int bh = blockIdx.y;
     const long long base = (long long)(bh / heads) * stride_b + (long long)(bh % heads) * stride_h;
-    const float *qrow = q + base + (long long)row * stride_s;
+    // in_map: q, k, v are in original order and physical row p lives at row in_map[p]
+    const float *qrow = q + base + (long long)(in_map ? in_map[row] : row) * stride_s;
     for (int d = lane; d < D; d += 32) sq[warp][d] = qrow[d];
     __syncwarp();
 
@@ -54,7 +55,8 @@ attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const
     for (int s = 0; s < n_seg; ++s) {
         const int end = seg_start[s] + seg_len[s];
         for (int j = seg_start[s] + lane; j < end; j += 32) {
-            const float4 *kj = reinterpret_cast<const float4 *>(k + base + (long long)j * stride_s);
+            const long long jrow = in_map ? in_map[j] : j;
+            const float4 *kj = reinterpret_cast<const float4 *>(k + base + jrow * stride_s);
             float dot = 0.f;
 #pragma unroll
             for (int d4 = 0; d4 < D / 4; ++d4) {
@@ -74,7 +76,7 @@ attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const
             }
             const float p = expf(x - m);
             l += p;
-            const float4 *vj = reinterpret_cast<const float4 *>(v + base + (long long)j * stride_s);
+            const float4 *vj = reinterpret_cast<const float4 *>(v + base + jrow * stride_s);
 #pragma unroll
             for (int d4 = 0; d4 < D / 4; ++d4) {
                 const float4 vv = __ldg(vj + d4);
@@ -111,7 +113,7 @@ attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const
 }
 
 int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, cudaStream_t stream) {
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream) {
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
     if ((bits & 15) || ((p->stride_b | p->stride_h | p->stride_s) & 3)) return HILBERTA_ERR_INVALID;
     dim3 grid((p->S + kRowsPerBlock - 1) / kRowsPerBlock, p->batch * p->heads);
@@ -120,7 +122,7 @@ int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, con
     case DD:                                                                                          \
         attn_fp32_kernel<DD><<<grid, block, 0, stream>>>(                                             \
             (const float *)q, (const float *)k, (const float *)v, (float *)out, p->stride_b,          \
-            p->stride_h, p->stride_s, p->heads, p->S, p->P, p->d_row_window, p->d_windows, out_map,   \
+            p->stride_h, p->stride_s, p->heads, p->S, p->P, p->d_row_window, p->d_windows, out_map, in_map,   \
             lse, p->scale);                                                                                \
         break;
     switch (p->head_dim) {

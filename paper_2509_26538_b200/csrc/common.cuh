@@ -104,10 +104,12 @@ namespace hilberta {
 // that physical row p goes to (the exit gather fused into the epilogue).
 // lse: nullptr, or [batch * heads, S] fp32 receiving log-sum-exp of the scaled logits
 // (natural log), indexed like `out` rows.
+// in_map: nullptr = q, k, v are in physical order; else they are in ORIGINAL order and physical
+// row p is read from row in_map[p] (the entry gather fused into the loads).
 int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, cudaStream_t stream);
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream);
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, cudaStream_t stream);
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream);
 int attn_bf16_prepare(hilberta_plan_t *p);
 int attn_bwd_prepare(hilberta_plan_t *p);
 // dq, dk, dv (bf16, physical order, the bound strides) from dout, q, k, v, out and the forward's lse.

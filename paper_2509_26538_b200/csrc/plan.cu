@@ -475,7 +475,7 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
 }
 
 static int forward_impl(const void *q, const void *k, const void *v, void *out, float *lse,
-                        const hilberta_plan_t *p, const int *out_map, void *stream) {
+                        const hilberta_plan_t *p, const int *out_map, const int *in_map, void *stream) {
     if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
     if (out == q || out == k || out == v) return HILBERTA_ERR_INVALID;
@@ -483,26 +483,32 @@ static int forward_impl(const void *q, const void *k, const void *v, void *out, 
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;  // the plan's tables live on another device
     cudaStream_t st = (cudaStream_t)stream;
-    if (p->dtype == HILBERTA_FP32) return launch_attn_fp32(p, q, k, v, out, lse, out_map, st);
+    if (p->dtype == HILBERTA_FP32) return launch_attn_fp32(p, q, k, v, out, lse, out_map, in_map, st);
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
     if (bits & 15) return HILBERTA_ERR_INVALID;
-    return launch_attn_bf16(p, q, k, v, out, lse, out_map, st);
+    return launch_attn_bf16(p, q, k, v, out, lse, out_map, in_map, st);
 }
 
 extern "C" int hilberta_forward(const void *q, const void *k, const void *v, void *out,
                                 const hilberta_plan_t *p, void *stream) {
-    return forward_impl(q, k, v, out, nullptr, p, nullptr, stream);
+    return forward_impl(q, k, v, out, nullptr, p, nullptr, nullptr, stream);
 }
 
 extern "C" int hilberta_forward_unpermute(const void *q, const void *k, const void *v, void *out,
                                           const hilberta_plan_t *p, void *stream) {
-    return forward_impl(q, k, v, out, nullptr, p, p ? p->d_phys2orig : nullptr, stream);
+    return forward_impl(q, k, v, out, nullptr, p, p ? p->d_phys2orig : nullptr, nullptr, stream);
+}
+
+extern "C" int hilberta_forward_fused(const void *q, const void *k, const void *v, void *out,
+                                      const hilberta_plan_t *p, int in_original, int out_original, void *stream) {
+    const int *map = p ? p->d_phys2orig : nullptr;
+    return forward_impl(q, k, v, out, nullptr, p, out_original ? map : nullptr, in_original ? map : nullptr, stream);
 }
 
 extern "C" int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out, float *lse,
                                     const hilberta_plan_t *p, void *stream) {
     if (!lse || ((uintptr_t)lse & 3)) return HILBERTA_ERR_INVALID;
-    return forward_impl(q, k, v, out, lse, p, nullptr, stream);
+    return forward_impl(q, k, v, out, lse, p, nullptr, nullptr, stream);
 }
 
 extern "C" int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
