@@ -535,8 +535,9 @@ extern "C" int hilberta_backward(const void *dout, const void *q, const void *k,
     return launch_attn_bwd(p, dout, q, k, v, out, lse, dq, dk, dv, p->d_delta, (cudaStream_t)stream);
 }
 
-// Whole path for host-resident activations: H2D copies, three entry gathers,
-// forward, exit gather, D2H copy.  Seven device buffers of one tensor each.
+// Whole path for host-resident activations: H2D copies, then ONE launch that reads q, k, v
+// through the permutation and writes `out` in the original order (entry and exit gathers
+// fused in), then the D2H copy.  Four device buffers of one tensor each.
 extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v, void *out,
                                      hilberta_plan_t *p, void *stream) {
     if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
@@ -547,29 +548,22 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
     const size_t esz = p->dtype == HILBERTA_BF16 ? 2 : 4;
     const size_t bytes = (size_t)p->batch * p->heads * p->S * p->head_dim * esz;
     const size_t slot = (bytes + 255) & ~(size_t)255;
-    if (p->ws_bytes < 7 * slot) {
+    if (p->ws_bytes < 4 * slot) {
         cudaFree(p->ws);
         p->ws = nullptr;
         p->ws_bytes = 0;
-        HB_CUDA(cudaMalloc(&p->ws, 7 * slot));
-        p->ws_bytes = 7 * slot;
+        HB_CUDA(cudaMalloc(&p->ws, 4 * slot));
+        p->ws_bytes = 4 * slot;
     }
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)p->ws;
     void *in[3] = {ws, ws + slot, ws + 2 * slot};
-    void *perm[3] = {ws + 3 * slot, ws + 4 * slot, ws + 5 * slot};
-    void *out_phys = ws + 6 * slot;
+    void *out_dev = ws + 3 * slot;
     const void *host_in[3] = {q, k, v};
-    const int bh = p->batch * p->heads;
-    for (int i = 0; i < 3; ++i) {
-        HB_CUDA(cudaMemcpyAsync(in[i], host_in[i], bytes, cudaMemcpyHostToDevice, st));
-        int rc = hilberta_permute(in[i], perm[i], p, bh, p->head_dim, p->dtype, st);
-        if (rc != HILBERTA_OK) return rc;
-    }
-    (void)bh;
-    int rc = hilberta_forward_unpermute(perm[0], perm[1], perm[2], out_phys, p, st);  // out_phys holds ORIGINAL order
+    for (int i = 0; i < 3; ++i) HB_CUDA(cudaMemcpyAsync(in[i], host_in[i], bytes, cudaMemcpyHostToDevice, st));
+    int rc = hilberta_forward_fused(in[0], in[1], in[2], out_dev, p, 1, 1, st);
     if (rc != HILBERTA_OK) return rc;
-    HB_CUDA(cudaMemcpyAsync(out, out_phys, bytes, cudaMemcpyDeviceToHost, st));
+    HB_CUDA(cudaMemcpyAsync(out, out_dev, bytes, cudaMemcpyDeviceToHost, st));
     HB_CUDA(cudaStreamSynchronize(st));
     return HILBERTA_OK;
 }

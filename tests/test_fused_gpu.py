@@ -63,3 +63,31 @@ def test_fused_strided_inputs():
         assert torch.equal(got.contiguous().view(torch.int16), want.view(torch.int16))
     finally:
         plan.destroy()
+
+
+@pytest.mark.parametrize("D,dtype", [(128, torch.bfloat16), (64, torch.float32)])
+def test_forward_host_matches_device_path(D, dtype):
+    """Host-buffer entry point (H2D, one fused launch, D2H) against permute -> forward -> unpermute."""
+    H = W = 32
+    nt, heads = 21, 2
+    S = nt + H * W
+    g = torch.Generator().manual_seed(79)
+    q, k, v = (torch.randn((1, heads, S, D), generator=g).to(dtype).pin_memory() for _ in range(3))
+    out_h = torch.empty_like(q).pin_memory()
+    plan = hb.Plan(H, W, 256, 192, 4, nt)
+    try:
+        qd, kd, vd = (t.cuda() for t in (q, k, v))
+        qp, kp, vp, op, od = (torch.empty_like(qd) for _ in range(5))
+        plan.bind_like(qd)
+        for src, dst in ((qd, qp), (kd, kp), (vd, vp)):
+            plan.permute(src, dst)
+        plan.forward(qp, kp, vp, op)
+        plan.unpermute(op, od)
+        for _ in range(2):   # the second call reuses the workspace
+            out_h.fill_(float("nan"))
+            plan.forward_host(q, k, v, out_h)
+            assert plan.status() == 0
+            view = torch.int16 if dtype == torch.bfloat16 else torch.int32
+            assert torch.equal(out_h.view(view), od.cpu().view(view))
+    finally:
+        plan.destroy()
