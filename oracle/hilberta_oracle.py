@@ -20,6 +20,10 @@ Where each piece comes from
   below (start at row 0 / col 0, end at row 0 / col W-1) is this build's
   reading.  Parity between the eight orientations is unpinned by the paper.
 * shared_cells : the fixed central region (Sec. 3.3).
+* hilbert3d_point and the `frames` arguments : Sec. 5 ("Extension to Video
+  Diffusion"): a 3-D Hilbert curve over (frame, row, col), tiles as contiguous
+  stretches of it, the same slide, and a central shared BOX.  The paper leaves
+  the curve and the box unspecified; both are this build's reading.
 * group_of : tile id of a Hilbert index at a given slide (Sec. 3.2, the
   formula for q_i(l)), read as "two tokens see each other iff their q_i(l)
   agree" -- the only reading that reproduces the ERF law of the same section.
@@ -77,22 +81,73 @@ def _log2_exact(n: int) -> int:
     return k
 
 
-def padded_side(H: int, W: int) -> int:
+def hilbert3d_point(d: int, k: int):
+    """Cell (frame, row, col) of index d on the 3-D Hilbert curve of a 2^k cube
+    (Sec. 5, "Extension to Video Diffusion": a three-dimensional Hilbert curve over
+    the spatio-temporal volume; the paper fixes no particular curve).
+
+    The curve used is the one of Skilling's transpose construction ("Programming
+    the Hilbert curve", 2004) with axes (frame, row, col): the 3k bits of d are
+    dealt round-robin to three k-bit words (most significant bit to the frame
+    word), the words are Gray-decoded, and the per-level exchanges / inversions
+    are undone from the finest level up.  Starts at (0, 0, 0).
+    """
+    X = [0, 0, 0]
+    for bit in range(3 * k):
+        if (d >> (3 * k - 1 - bit)) & 1:
+            X[bit % 3] |= 1 << (k - 1 - bit // 3)
+    if k == 0:
+        return (0, 0, 0)
+    t = X[2] >> 1
+    X[2] ^= X[1]
+    X[1] ^= X[0]
+    X[0] ^= t
+    Q = 2
+    while Q != (1 << k):
+        Pm = Q - 1
+        for i in (2, 1, 0):
+            if X[i] & Q:
+                X[0] ^= Pm
+            else:
+                t = (X[0] ^ X[i]) & Pm
+                X[0] ^= t
+                X[i] ^= t
+        Q <<= 1
+    return (X[0], X[1], X[2])
+
+
+def padded_side(H: int, W: int, frames: int = 1) -> int:
     """Side n = 2^k of the smallest enclosing power-of-two square (Appendix "Hilbert
     Curve for General Shape": the curve is built on an enclosing regular grid and the
-    H x W sub-region is extracted; cells outside it are padding)."""
-    if H < 1 or W < 1:
+    H x W sub-region is extracted; cells outside it are padding).  With frames > 1
+    the enclosing shape is a cube that also holds the frame axis."""
+    if H < 1 or W < 1 or frames < 1:
         raise ValueError("empty grid")
     n = 1
-    while n < max(H, W):
+    while n < max(H, W, frames if frames > 1 else 1):
         n *= 2
     return n
 
 
-def hilbert_cell_index(H: int, W: int) -> np.ndarray:
+def padded_length(H: int, W: int, frames: int = 1) -> int:
+    """Length of the padded curve: n^2 for an image, n^3 for a video volume."""
+    n = padded_side(H, W, frames)
+    return n * n if frames == 1 else n * n * n
+
+
+def hilbert_cell_index(H: int, W: int, frames: int = 1) -> np.ndarray:
     """row-major cell id r*W + c -> Hilbert index of the cell on the padded n x n grid.
-    int32[HW].  For a power-of-two square this is pi^-1 itself."""
-    n = padded_side(H, W)
+    int32[HW].  For a power-of-two square this is pi^-1 itself.  With frames > 1:
+    cell id (f*H + r)*W + c -> index on the 3-D curve of the padded cube."""
+    n = padded_side(H, W, frames)
+    if frames > 1:
+        k = _log2_exact(n)
+        out = np.empty(frames * H * W, dtype=np.int32)
+        for d in range(n * n * n):
+            f, y, x = hilbert3d_point(d, k)
+            if f < frames and y < H and x < W:
+                out[(f * H + y) * W + x] = d
+        return out
     pts = hilbert_points(_log2_exact(n))
     out = np.empty(H * W, dtype=np.int32)
     for d, (x, y) in enumerate(pts):
@@ -101,15 +156,15 @@ def hilbert_cell_index(H: int, W: int) -> np.ndarray:
     return out
 
 
-def hilbert_d2t(H: int, W: int) -> np.ndarray:
+def hilbert_d2t(H: int, W: int, frames: int = 1) -> np.ndarray:
     """d -> row-major cell id r*W + c (pi of Sec. 3.1). int32[HW].  On a general
     shape d is the RANK of the cell among the real cells in padded-curve order."""
-    return np.argsort(hilbert_cell_index(H, W), kind="stable").astype(np.int32)
+    return np.argsort(hilbert_cell_index(H, W, frames), kind="stable").astype(np.int32)
 
 
-def hilbert_t2d(H: int, W: int) -> np.ndarray:
+def hilbert_t2d(H: int, W: int, frames: int = 1) -> np.ndarray:
     """row-major cell id -> Hilbert index d (pi^-1; rank on a general shape). int32[HW]."""
-    d2t = hilbert_d2t(H, W)
+    d2t = hilbert_d2t(H, W, frames)
     t2d = np.empty_like(d2t)
     t2d[d2t] = np.arange(d2t.size, dtype=np.int32)
     return t2d
@@ -120,9 +175,24 @@ def hilbert_t2d(H: int, W: int) -> np.ndarray:
 # --------------------------------------------------------------------------
 
 
-def shared_cells(H: int, W: int, shared_region: int) -> np.ndarray:
-    """Row-major ids of the centred shared_region x shared_region block."""
+def shared_cells(H: int, W: int, shared_region: int, frames: int = 1, shared_frames: int = 0) -> np.ndarray:
+    """Row-major ids of the centred shared_region x shared_region block.  For a video
+    volume (frames > 1) the region is the centred box of shared_frames frames by
+    shared_region x shared_region cells ("shared anchors ... also along the temporal
+    dimension", Sec. 5)."""
     hs = int(shared_region)
+    if frames > 1:
+        fs = int(shared_frames)
+        if hs == 0 or fs == 0:
+            if hs or fs:
+                raise ValueError("a shared box needs both extents")
+            return np.zeros(0, dtype=np.int32)
+        if hs < 0 or hs > H or hs > W or hs % 2 or fs < 0 or fs > frames or fs % 2:
+            raise ValueError("shared box extents must be even and fit the volume")
+        f0, r0, c0 = frames // 2 - fs // 2, H // 2 - hs // 2, W // 2 - hs // 2
+        cells = [(f * H + r) * W + c for f in range(f0, f0 + fs) for r in range(r0, r0 + hs)
+                 for c in range(c0, c0 + hs)]
+        return np.array(cells, dtype=np.int32)
     if hs == 0:
         return np.zeros(0, dtype=np.int32)
     if hs < 0 or hs > H or hs > W or hs % 2:
@@ -133,10 +203,10 @@ def shared_cells(H: int, W: int, shared_region: int) -> np.ndarray:
     return np.array(cells, dtype=np.int32)
 
 
-def shared_hilbert_indices(H: int, W: int, shared_region: int) -> np.ndarray:
+def shared_hilbert_indices(H: int, W: int, shared_region: int, frames: int = 1, shared_frames: int = 0) -> np.ndarray:
     """Sorted (padded) Hilbert indices of the shared cells."""
-    pidx = hilbert_cell_index(H, W)
-    return np.sort(pidx[shared_cells(H, W, shared_region)]).astype(np.int32)
+    pidx = hilbert_cell_index(H, W, frames)
+    return np.sort(pidx[shared_cells(H, W, shared_region, frames, shared_frames)]).astype(np.int32)
 
 
 # --------------------------------------------------------------------------
@@ -153,7 +223,7 @@ def group_of(d, layer_offset: int, HW: int, tile: int):
     return ((d + int(layer_offset)) // tile) % T
 
 
-def token_classes(H, W, tile, layer_offset, shared_region, n_text):
+def token_classes(H, W, tile, layer_offset, shared_region, n_text, frames=1, shared_frames=0):
     """Per original token: is_global (uint8[S]) and group (int32[S], -1 = text).
 
     Text tokens and shared-region tokens are global (Appendix A / Sec. 3.3);
@@ -162,25 +232,24 @@ def token_classes(H, W, tile, layer_offset, shared_region, n_text):
     stay in the sequence and are masked out, as the appendix says), so `tile`
     must divide the padded length n*n.
     """
-    HW = H * W
+    HW = frames * H * W
     S = n_text + HW
-    n = padded_side(H, W)
-    pidx = hilbert_cell_index(H, W)
+    pidx = hilbert_cell_index(H, W, frames)
     is_global = np.zeros(S, dtype=np.uint8)
     is_global[:n_text] = 1
-    is_global[n_text + shared_cells(H, W, shared_region)] = 1
+    is_global[n_text + shared_cells(H, W, shared_region, frames, shared_frames)] = 1
     group = np.full(S, -1, dtype=np.int32)
-    group[n_text:] = group_of(pidx, layer_offset, n * n, tile).astype(np.int32)
+    group[n_text:] = group_of(pidx, layer_offset, padded_length(H, W, frames), tile).astype(np.int32)
     return is_global, group
 
 
-def mask(H, W, tile, layer_offset, shared_region, n_text) -> np.ndarray:
+def mask(H, W, tile, layer_offset, shared_region, n_text, frames=1, shared_frames=0) -> np.ndarray:
     """Boolean S x S mask over original token indices.
 
     M[i,j] = 1 iff i is global, or j is global, or i and j are image tokens
     of the same slid tile.
     """
-    is_global, group = token_classes(H, W, tile, layer_offset, shared_region, n_text)
+    is_global, group = token_classes(H, W, tile, layer_offset, shared_region, n_text, frames, shared_frames)
     g = is_global.astype(bool)
     img = group >= 0
     same = (group[:, None] == group[None, :]) & img[:, None] & img[None, :]
@@ -194,13 +263,13 @@ def mask_row(i, is_global, group) -> np.ndarray:
     return is_global.astype(bool) | ((group == group[i]) & (group >= 0))
 
 
-def nnz(H, W, tile, layer_offset, shared_region, n_text) -> int:
+def nnz(H, W, tile, layer_offset, shared_region, n_text, frames=1, shared_frames=0) -> int:
     """Number of ones in the mask, as the sum of the row counts."""
-    is_global, group = token_classes(H, W, tile, layer_offset, shared_region, n_text)
+    is_global, group = token_classes(H, W, tile, layer_offset, shared_region, n_text, frames, shared_frames)
     S = is_global.size
     n_global = int(is_global.sum())
     nonshared_img = (group >= 0) & (is_global == 0)
-    T = (padded_side(H, W) ** 2) // tile
+    T = padded_length(H, W, frames) // tile
     per_group = np.bincount(group[nonshared_img], minlength=T).astype(np.int64)
     total = n_global * S
     # a non-global row sees every global column plus the non-global members of its tile
@@ -303,7 +372,7 @@ def attention_backward(q, k, v, M, dout, scale=None):
 # --------------------------------------------------------------------------
 
 
-def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
+def plan_arrays(H, W, tile, layer_offset, shared_region, n_text, frames=1, shared_frames=0) -> dict:
     """Canonical integer arrays a plan must reproduce bit for bit.
 
     physical order = [text | shared image tokens by ascending Hilbert index |
@@ -315,17 +384,17 @@ def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
     physical ranges.  seg0 is the range that starts at lo.  Empty ranges are (0, 0).
     shared_runs are maximal runs of shared (padded) Hilbert indices.
     """
-    HW = H * W
+    HW = frames * H * W
     S = n_text + HW
-    n = padded_side(H, W)
-    NP = n * n
+    n = padded_side(H, W, frames)
+    NP = padded_length(H, W, frames)
     if tile < 1 or NP % tile:
         raise ValueError("tile must divide the (padded) curve length")
     T = NP // tile
-    d2t = hilbert_d2t(H, W)
-    t2d = hilbert_t2d(H, W)
-    pidx = hilbert_cell_index(H, W)                      # cell -> padded index
-    sh_cells = shared_cells(H, W, shared_region)
+    d2t = hilbert_d2t(H, W, frames)
+    t2d = hilbert_t2d(H, W, frames)
+    pidx = hilbert_cell_index(H, W, frames)              # cell -> padded index
+    sh_cells = shared_cells(H, W, shared_region, frames, shared_frames)
     sh = np.sort(pidx[sh_cells]).astype(np.int32)        # shared padded indices
     n_sh = sh.size
     P = n_text + n_sh
@@ -374,7 +443,7 @@ def plan_arrays(H, W, tile, layer_offset, shared_region, n_text) -> dict:
         "orig2phys": orig2phys,
         "shared_runs": shared_runs,
         "windows": windows,
-        "nnz": nnz(H, W, tile, layer_offset, shared_region, n_text),
+        "nnz": nnz(H, W, tile, layer_offset, shared_region, n_text, frames, shared_frames),
         "n_shared": int(n_sh),
         "prefix": int(P),
         "padded_side": int(n),
