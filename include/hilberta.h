@@ -67,7 +67,7 @@ extern "C" {
 #define HILBERTA_EXPORT_SHARED_RUNS 4 /* int32[n][2] maximal runs (start, length) of shared positions on the padded curve */
 #define HILBERTA_EXPORT_WINDOWS 5     /* int32[T][5] per slid tile: lo, seg0_start, seg0_len, seg1_start, seg1_len */
 #define HILBERTA_EXPORT_NNZ 6         /* uint64[1]   number of (query, key) pairs the mask keeps */
-#define HILBERTA_EXPORT_INFO 7        /* int32[9]    H, W, tile, offset mod NP, shared_region, n_text, n_shared, T, padded side n */
+#define HILBERTA_EXPORT_INFO 7        /* int32[11]   H, W, tile, offset mod NP, shared_region, n_text, n_shared, T, padded side n, frames, shared_frames */
 
 typedef struct hilberta_plan_s hilberta_plan_t;
 
@@ -110,6 +110,20 @@ int hilberta_plan(int H, int W, int tile, int layer_offset, int shared_region, i
  * region at 1024^2: groups of 960 or 240 tokens). */
 int hilberta_plan_groups(int H, int W, int groups, int layer_offset, int shared_region, int n_text,
                          hilberta_plan_t **out);
+
+/* The plan for a video volume (Sec. 5, "Extension to Video Diffusion"): `frames` x H x W
+ * tokens, original order [text | (f * H + r) * W + c], reordered along a THREE-dimensional
+ * Hilbert curve so that a tile is a compact spatio-temporal block; tiles, slide and
+ * wrap-around are those of hilberta_plan on that curve.  The paper names the idea and fixes
+ * neither the curve nor the shared region; this library uses the curve of Skilling's
+ * transpose construction with axes (frame, row, col), starting at cell (0, 0, 0), on the
+ * smallest enclosing power-of-two cube (side n >= max(frames, H, W); cells outside the volume
+ * are padding, as for general image shapes; `tile` must divide n^3), and a centred shared BOX
+ * of shared_frames x shared_region x shared_region cells (both even, both zero for none).
+ * frames >= 2; frames, H, W <= 128.  Everything downstream (export, bind, forward,
+ * backward, permute) is unchanged: the kernels only ever see contiguous physical ranges. */
+int hilberta_plan_video(int frames, int H, int W, int tile, int layer_offset, int shared_region,
+                        int shared_frames, int n_text, hilberta_plan_t **out);
 
 /* Free a plan and every device table it owns.  NULL is accepted. */
 int hilberta_plan_destroy(hilberta_plan_t *plan);

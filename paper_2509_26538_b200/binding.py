@@ -23,7 +23,7 @@ BF16, FP32 = 0, 1
 
 # every symbol include/hilberta.h declares
 SYMBOLS = (
-    "hilberta_plan", "hilberta_plan_groups", "hilberta_plan_destroy", "hilberta_plan_export",
+    "hilberta_plan", "hilberta_plan_groups", "hilberta_plan_video", "hilberta_plan_destroy", "hilberta_plan_export",
     "hilberta_plan_bind",
     "hilberta_forward", "hilberta_forward_unpermute", "hilberta_forward_fused", "hilberta_forward_lse",
     "hilberta_backward",
@@ -61,6 +61,8 @@ def lib():
     L.hilberta_plan.restype = i32
     L.hilberta_plan_groups.argtypes = [i32] * 6 + [ctypes.POINTER(vp)]
     L.hilberta_plan_groups.restype = i32
+    L.hilberta_plan_video.argtypes = [i32] * 8 + [ctypes.POINTER(vp)]
+    L.hilberta_plan_video.restype = i32
     L.hilberta_plan_destroy.argtypes = [vp]
     L.hilberta_plan_destroy.restype = i32
     L.hilberta_plan_export.argtypes = [vp, i32, vp, sz, ctypes.POINTER(sz)]
@@ -133,17 +135,22 @@ _EXPORT_NP = {
 class Plan:
     """Owner of a hilberta_plan_t*.  Methods mirror the C entry points."""
 
-    def __init__(self, H, W, tile, layer_offset, shared_region, n_text, groups=0):
-        """tile > 0: hilberta_plan; groups > 0 (tile ignored): hilberta_plan_groups."""
+    def __init__(self, H, W, tile, layer_offset, shared_region, n_text, groups=0, frames=1, shared_frames=0):
+        """tile > 0: hilberta_plan; groups > 0 (tile ignored): hilberta_plan_groups;
+        frames > 1: hilberta_plan_video (a frames x H x W volume)."""
         self._h = ctypes.c_void_p()
-        if groups:
+        if frames > 1:
+            _check(lib().hilberta_plan_video(int(frames), int(H), int(W), int(tile), int(layer_offset),
+                                             int(shared_region), int(shared_frames), int(n_text),
+                                             ctypes.byref(self._h)), "hilberta_plan_video")
+        elif groups:
             _check(lib().hilberta_plan_groups(int(H), int(W), int(groups), int(layer_offset), int(shared_region),
                                               int(n_text), ctypes.byref(self._h)), "hilberta_plan_groups")
         else:
             _check(lib().hilberta_plan(int(H), int(W), int(tile), int(layer_offset), int(shared_region),
                                        int(n_text), ctypes.byref(self._h)), "hilberta_plan")
         self.H, self.W, self.tile, self.n_text = int(H), int(W), int(tile), int(n_text)
-        self.S = int(n_text) + int(H) * int(W)
+        self.S = int(n_text) + int(frames) * int(H) * int(W)
         self._bound = None
 
     @property

@@ -57,6 +57,61 @@ __global__ void hilbert_lut_kernel(int k, int H, int W, int *__restrict__ cell_o
     }
 }
 
+// Video volumes (Sec. 5, "Extension to Video Diffusion"): one thread per cell of the padded
+// n x n x n cube, axes (frame, row, col).  The cell's index on the 3-D Hilbert curve comes from
+// the coordinate -> index direction of Skilling's transpose construction: per level, from the top
+// bit down, an inversion or an exchange against axis 0; then a Gray encoding across the axes; the
+// index is the bit interleave of the three resulting words (frame word most significant).
+__global__ void hilbert3d_lut_kernel(int k, int F, int H, int W, int *__restrict__ cell_of_pd,
+                                     int *__restrict__ pd_of_cell, unsigned char *__restrict__ kind_by_pd,
+                                     int sh_f0, int sh_r0, int sh_c0, int sh_side, int sh_frames) {
+    const int n = 1 << k;
+    const int pc = blockIdx.x * blockDim.x + threadIdx.x;   // padded cell
+    if (pc >= n * n * n) return;
+    const int f = pc >> (2 * k), row = (pc >> k) & (n - 1), col = pc & (n - 1);
+    unsigned X0 = f, X1 = row, X2 = col;
+    for (unsigned Q = 1u << (k - 1); Q > 1; Q >>= 1) {
+        const unsigned Pm = Q - 1;
+        if (X0 & Q) X0 ^= Pm;                 // axis 0 against itself: inversion only
+        if (X1 & Q) {
+            X0 ^= Pm;
+        } else {
+            const unsigned t = (X0 ^ X1) & Pm;
+            X0 ^= t;
+            X1 ^= t;
+        }
+        if (X2 & Q) {
+            X0 ^= Pm;
+        } else {
+            const unsigned t = (X0 ^ X2) & Pm;
+            X0 ^= t;
+            X2 ^= t;
+        }
+    }
+    X1 ^= X0;
+    X2 ^= X1;
+    unsigned t = 0;
+    for (unsigned Q = 1u << (k - 1); Q > 1; Q >>= 1)
+        if (X2 & Q) t ^= Q - 1;
+    X0 ^= t;
+    X1 ^= t;
+    X2 ^= t;
+    int d = 0;
+    for (int b = k - 1; b >= 0; --b)
+        d = (d << 3) | (int)(((X0 >> b) & 1) << 2 | ((X1 >> b) & 1) << 1 | ((X2 >> b) & 1));
+    if (f < F && row < H && col < W) {
+        const int cell = (f * H + row) * W + col;
+        pd_of_cell[cell] = d;
+        cell_of_pd[d] = cell;
+        const bool sh = f >= sh_f0 && f < sh_f0 + sh_frames && row >= sh_r0 && row < sh_r0 + sh_side &&
+                        col >= sh_c0 && col < sh_c0 + sh_side;
+        kind_by_pd[d] = sh ? CELL_SHARED : CELL_REAL;
+    } else {
+        cell_of_pd[d] = -1;
+        kind_by_pd[d] = CELL_PAD;
+    }
+}
+
 // c_ns[d] = number of real non-shared cells with padded index below d, c_real[d] =
 // number of real cells below d, for d in [0, NP].  Single block; each thread owns a
 // contiguous slice.
@@ -244,8 +299,13 @@ static int build_plan(hilberta_plan_t *p) {
             rc = HILBERTA_ERR_CUDA;
             break;
         }
-        hilbert_lut_kernel<<<(NP + 255) / 256, 256>>>(p->k_log2, p->H, p->W, d_cell_of_pd, d_pd_of_cell, d_kind,
-                                                      sh_r0, sh_c0, p->shared_region);
+        if (p->frames > 1)
+            hilbert3d_lut_kernel<<<(NP + 255) / 256, 256>>>(p->k_log2, p->frames, p->H, p->W, d_cell_of_pd,
+                                                            d_pd_of_cell, d_kind, p->frames / 2 - p->shared_frames / 2,
+                                                            sh_r0, sh_c0, p->shared_region, p->shared_frames);
+        else
+            hilbert_lut_kernel<<<(NP + 255) / 256, 256>>>(p->k_log2, p->H, p->W, d_cell_of_pd, d_pd_of_cell, d_kind,
+                                                          sh_r0, sh_c0, p->shared_region);
         g_launches.fetch_add(1);
         cell_scan_kernel<<<1, 1024>>>(d_kind, NP, p->d_c, d_c_real);
         g_launches.fetch_add(1);
@@ -315,21 +375,35 @@ using namespace hilberta;
 
 // tile > 0: curve tiling (tiles of `tile` positions of the padded curve).
 // groups > 0: compact tiling (Algorithm 1's equal groups over the non-shared tokens).
-static int make_plan(int H, int W, int tile, int groups, int layer_offset, int shared_region, int n_text,
-                     hilberta_plan_t **out) {
+// frames > 1: a video volume of `frames` x H x W cells on the 3-D curve of the padded cube, with a
+// central shared box of shared_frames x shared_region x shared_region cells.
+static int make_plan(int frames, int H, int W, int tile, int groups, int layer_offset, int shared_region,
+                     int shared_frames, int n_text, hilberta_plan_t **out) {
     if (!out) return HILBERTA_ERR_INVALID;
     *out = nullptr;
     const bool compact = groups > 0;
-    if (H < 1 || W < 1 || n_text < 0 || shared_region < 0) return HILBERTA_ERR_INVALID;
+    if (frames < 1 || H < 1 || W < 1 || n_text < 0 || shared_region < 0 || shared_frames < 0)
+        return HILBERTA_ERR_INVALID;
     if (!compact && tile < 1) return HILBERTA_ERR_INVALID;
     if (H > 1024 || W > 1024) return HILBERTA_ERR_UNSUPPORTED;
-    const int HW = H * W;
-    int k_log2 = 0;                       // padded side n = 2^k >= max(H, W)
-    while ((1 << k_log2) < (H > W ? H : W)) ++k_log2;
-    const int NP = 1 << (2 * k_log2);     // length of the padded curve
+    if (frames > 1 && (H > 128 || W > 128 || frames > 128)) return HILBERTA_ERR_UNSUPPORTED;
+    const int HW = frames * H * W;        // grid cells = image (or video) tokens
+    int side = H > W ? H : W;
+    if (frames > 1 && frames > side) side = frames;
+    int k_log2 = 0;                       // padded side n = 2^k >= max(H, W[, frames])
+    while ((1 << k_log2) < side) ++k_log2;
+    if (frames > 1 && k_log2 < 1) k_log2 = 1;
+    const int NP = 1 << ((frames > 1 ? 3 : 2) * k_log2);   // length of the padded curve
     if (shared_region % 2 || shared_region > H || shared_region > W) return HILBERTA_ERR_INVALID;
+    if (frames > 1) {
+        if (shared_frames % 2 || shared_frames > frames) return HILBERTA_ERR_INVALID;
+        if ((shared_frames == 0) != (shared_region == 0)) return HILBERTA_ERR_INVALID;  // a box needs both extents
+    } else {
+        shared_frames = 1;
+    }
     if ((long long)n_text + HW > (1ll << 30)) return HILBERTA_ERR_INVALID;
-    const int R = HW - shared_region * shared_region;   // non-shared image tokens
+    const int n_shared = shared_region * shared_region * shared_frames;
+    const int R = HW - n_shared;          // non-shared image tokens
     if (compact) {
         if (R < 1 || R % groups) return HILBERTA_ERR_INVALID;
         tile = R / groups;
@@ -347,6 +421,8 @@ static int make_plan(int H, int W, int tile, int groups, int layer_offset, int s
     if (!p) return HILBERTA_ERR_NOMEM;
     p->device = dev;
     p->sm_count = prop.multiProcessorCount;
+    p->frames = frames;
+    p->shared_frames = frames > 1 ? shared_frames : 0;
     p->H = H;
     p->W = W;
     p->HW = HW;
@@ -360,7 +436,7 @@ static int make_plan(int H, int W, int tile, int groups, int layer_offset, int s
     p->offset = (int)o;
     p->shared_region = shared_region;
     p->n_text = n_text;
-    p->n_shared = shared_region * shared_region;
+    p->n_shared = n_shared;
     p->T = compact ? groups : NP / tile;
     p->S = n_text + HW;
     p->P = n_text + p->n_shared;
@@ -380,7 +456,7 @@ extern "C" int hilberta_plan(int H, int W, int tile, int layer_offset, int share
         if (out) *out = nullptr;
         return HILBERTA_ERR_INVALID;
     }
-    return make_plan(H, W, tile, 0, layer_offset, shared_region, n_text, out);
+    return make_plan(1, H, W, tile, 0, layer_offset, shared_region, 0, n_text, out);
 }
 
 extern "C" int hilberta_plan_groups(int H, int W, int groups, int layer_offset, int shared_region, int n_text,
@@ -389,7 +465,16 @@ extern "C" int hilberta_plan_groups(int H, int W, int groups, int layer_offset, 
         if (out) *out = nullptr;
         return HILBERTA_ERR_INVALID;
     }
-    return make_plan(H, W, 0, groups, layer_offset, shared_region, n_text, out);
+    return make_plan(1, H, W, 0, groups, layer_offset, shared_region, 0, n_text, out);
+}
+
+extern "C" int hilberta_plan_video(int frames, int H, int W, int tile, int layer_offset, int shared_region,
+                                   int shared_frames, int n_text, hilberta_plan_t **out) {
+    if (tile < 1 || frames < 2) {
+        if (out) *out = nullptr;
+        return HILBERTA_ERR_INVALID;
+    }
+    return make_plan(frames, H, W, tile, 0, layer_offset, shared_region, shared_frames, n_text, out);
 }
 
 extern "C" int hilberta_plan_destroy(hilberta_plan_t *plan) {
@@ -420,7 +505,8 @@ extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *ho
             break;
         case HILBERTA_EXPORT_NNZ: need = sizeof(uint64_t); hsrc = &nnz; break;
         case HILBERTA_EXPORT_INFO:
-            tmp = {p->H, p->W, p->tile, p->offset, p->shared_region, p->n_text, p->n_shared, p->T, 1 << p->k_log2};
+            tmp = {p->H, p->W, p->tile, p->offset, p->shared_region, p->n_text, p->n_shared, p->T, 1 << p->k_log2,
+                   p->frames, p->shared_frames};
             need = sizeof(int) * tmp.size();
             hsrc = tmp.data();
             break;

@@ -23,7 +23,7 @@ def _check(H, tile, o, hs, nt, W=None):
         assert int(plan.export(hb.EXPORT_NNZ)[0]) == ref["nnz"]
         info = plan.export(hb.EXPORT_INFO).tolist()
         NP = orc.padded_side(H, W) ** 2
-        assert info == [H, W, tile, o % NP, hs, nt, hs * hs, NP // tile, orc.padded_side(H, W)]
+        assert info == [H, W, tile, o % NP, hs, nt, hs * hs, NP // tile, orc.padded_side(H, W), 1, 0]
     finally:
         plan.destroy()
 
