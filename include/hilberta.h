@@ -194,9 +194,9 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  *                      not alias each other or any input.  Every row is written.
  * All pointers 16-byte aligned (lse: 4).  Asynchronous on `stream`; three kernel
  * launches; no allocation, no synchronisation.  A per-row scratch array
- * (batch * heads * S floats, owned by the plan, allocated by hilberta_plan_bind)
- * carries delta between the launches, so two backward calls on the same plan
- * must not overlap on the device.
+ * (2 * batch * heads * S floats, owned by the plan, allocated by hilberta_plan_bind)
+ * carries lse * log2(e) and delta between the launches, so two backward calls on
+ * the same plan must not overlap on the device.
  *
  * Errors: ERR_INVALID (NULL, misaligned or aliasing pointers, wrong device),
  * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding: only the bf16 tensor-core path has a
@@ -208,8 +208,8 @@ int hilberta_backward(const void *dout, const void *q, const void *k, const void
 /* hilberta_backward for callers that must not allocate.  (The paper has no
  * counterpart: this is a deployment variant of the call above.)
  *
- * hilberta_backward keeps its per-row scratch (delta, one float per batch, head
- * and token) in memory that hilberta_plan_bind obtains from cudaMalloc, once per
+ * hilberta_backward keeps its per-row scratch (two floats per batch, head and
+ * token) in memory that hilberta_plan_bind obtains from cudaMalloc, once per
  * plan.  Some hosts cannot afford that: a serving process that handed all device
  * memory to its own pool at start-up, so that a later cudaMalloc fails; a
  * latency-bound loop that must avoid the device-wide synchronisation an
@@ -221,9 +221,9 @@ int hilberta_backward(const void *dout, const void *q, const void *k, const void
  *
  * Arguments, layouts, alignment, results and errors are those of
  * hilberta_backward, and the output is the same.  In addition:
- *   - batch * heads * S  >  HILBERTA_STATIC_SCRATCH_FLOATS  ->  ERR_BUFFER, nothing
- *     is launched (the Flux shapes at 1024^2 and 2048^2 fit; 4096^2 with 24 heads
- *     does not: use hilberta_backward there);
+ *   - 2 * batch * heads * S  >  HILBERTA_STATIC_SCRATCH_FLOATS  ->  ERR_BUFFER,
+ *     nothing is launched (the Flux shapes at 1024^2 and 2048^2 fit; 4096^2 with 24
+ *     heads does not: use hilberta_backward there);
  *   - the call itself performs no cudaMalloc, cudaFree or other allocation;
  *   - the FIRST call on each device looks up the array's device address (with
  *     that device current) and caches it; make that first call before any stream

@@ -7,20 +7,19 @@
 // With P = exp(s Q K^T - LSE), dP = dO V^T, delta = rowsum(dO * O) and
 // dS = P * (dP - delta):   dQ = s dS K,   dK = s dS^T Q,   dV = P^T dO.
 //
-// Three launches: a bandwidth-bound pass that writes delta, then one tensor-core
-// kernel in two modes that share all code but the element-wise step.
+// Three launches: a bandwidth-bound pass that writes (LSE * log2 e, delta) per row,
+// then one tensor-core kernel in two modes that share all code but a few lines.
 //   mode DQ : resident tile = 128 query rows (Q_i, dO_i); streamed = their keys (K_j, V_j)
-//             acc1 = Q_i K_j^T, acc2 = dO_i V_j^T, dS -> TMEM, dQ_i += dS K_j
+//             A = Q_i K_j^T, B = dO_i V_j^T, dS -> TMEM, dQ_i += dS K_j
 //   mode DKV: resident tile = 128 key rows (K_j, V_j); streamed = the queries that see them
-//             acc1 = K_j Q_i^T, acc2 = V_j dO_i^T (transposed scores: a thread owns a KEY row),
+//             A = K_j Q_i^T, B = V_j dO_i^T (transposed scores: a thread owns a KEY row),
 //             P^T, dS^T -> TMEM, dV_j += P^T dO_i, dK_j += dS^T Q_i
-// Streamed rows come in sub-blocks of 64 with two accumulator buffers, so the MMAs of
-// sub-block s + 1 run while the CUDA cores work on sub-block s; the two element-wise
-// warpgroups each take 32 of the 64 columns of every sub-block, which halves the
-// latency of the MMA -> element-wise -> MMA chain.  TMEM: acc1/acc2 of buffer b at
-// [128 b, +64) and [128 b + 64, +64); P and dS (bf16) overwrite them in place, each
-// warpgroup inside the columns it has just read.  DKV: two buffers, dK at [256, 384),
-// dV at [384, 512).  DQ: three buffers (the MMAs run two sub-blocks ahead), dQ at [384, 512).
+// Streamed rows come in blocks of 128.  TMEM: region A (scores, 128 columns), region B (dP,
+// 128 columns), outputs.  The element-wise step works in two phases: phase 1 turns the scores
+// into weights as soon as A is written and releases A at once, so the scores of the NEXT block
+// are computed while phase 2 (which needs B) and the output MMAs of this block run; phase 2
+// overwrites B in place with P and dS (bf16), each thread inside the 32 columns it has just
+// read.  Per block the tensor pipe sees  A(s+1) | out(s) | B(s+1)  back to back.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -28,6 +27,7 @@
 #include <functional>
 #include <mutex>
 #include <queue>
+#include <type_traits>
 #include <utility>
 
 #include "common.cuh"
@@ -41,36 +41,35 @@ int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, 
 namespace {
 
 constexpr int BM = 128;   // resident rows per work item
-constexpr int SUB = 64;   // streamed rows per sub-block
+constexpr int BK = 128;   // streamed rows per block
 constexpr int HD = 128;
-constexpr int NST_MAX = 5;   // ring of streamed sub-blocks (two 16-KB tiles each): 5 slots in DQ mode, 4 in DKV
-#ifndef HB_NST_DQ
-#define HB_NST_DQ 5
-#endif
-#ifndef HB_NST_DKV
-#define HB_NST_DKV 4
-#endif
-__host__ __device__ constexpr int nst_of(int mode) { return mode == 0 ? HB_NST_DQ : HB_NST_DKV; }
-constexpr int RES_BYTES = BM * HD * 2;        // 32 KB: two 64-column slabs of 128 rows
-constexpr int RES_SLAB = RES_BYTES / 2;
-constexpr int SUBT_BYTES = SUB * HD * 2;      // 16 KB: two 64-column slabs of 64 rows
-constexpr int SUBT_SLAB = SUBT_BYTES / 2;
-constexpr int STAGE_BYTES = 2 * SUBT_BYTES;
+constexpr int TILE_BYTES = BM * HD * 2;   // 32 KB: two 64-column slabs of 128 rows
+constexpr int SLAB_BYTES = TILE_BYTES / 2;
+constexpr int NT1 = 3;    // ring of the streamed operand that is read twice (scores early, output MMA late)
+constexpr int NT2 = 2;    // ring of the streamed operand of dP
+constexpr int STAT_BYTES = 2 * BK * 4;      // lse2[128] then delta[128] of a block's streamed rows (DKV)
 constexpr int THREADS = 512;  // 8 element-wise warps, 4 single-lane service warps, 4 epilogue warps
-// accumulator buffers: DQ has TMEM for three (its output needs 128 columns), DKV for two
-__host__ __device__ constexpr int nb_of(int mode) { return mode == 0 ? 3 : 2; }
-__host__ __device__ constexpr int smem_bytes_of(int mode) { return 2 * RES_BYTES + nst_of(mode) * STAGE_BYTES + 1024; }
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int MODE_DQ = 0, MODE_DKV = 1;
 
 enum Bar {
     RES_FULL = 0, RES_EMPTY, OUT_FULL, EPI_DONE, DRAIN,
-    S_FULL,                      // [NB] acc1 / acc2 of buffer b written
-    P_READY = S_FULL + 3,        // [NB] P / dS of buffer b written, 256 arrivals
-    ST_FULL = P_READY + 3, ST_EMPTY = ST_FULL + NST_MAX,
-    STAT_FULL = ST_EMPTY + NST_MAX,   // DKV: statistics of the streamed rows of ring slot s written
-    NUM_BARS = STAT_FULL + NST_MAX
+    S_FULL,       // region A written
+    A_DONE,       // region A read by every element-wise thread (256 arrivals)
+    DP_FULL,      // region B written
+    P_READY,      // P / dS written over region B (256 arrivals)
+    T1_FULL, T1_EMPTY = T1_FULL + NT1,
+    T2_FULL = T1_EMPTY + NT1, T2_EMPTY = T2_FULL + NT2,
+    NUM_BARS = T2_EMPTY + NT2
 };
+
+// shared memory map (all dynamic; the tile area must start on a 1024-byte boundary)
+constexpr int OFF_R1 = 0, OFF_R2 = TILE_BYTES, OFF_T1 = 2 * TILE_BYTES, OFF_T2 = OFF_T1 + NT1 * TILE_BYTES;
+constexpr int OFF_STAT = OFF_T2 + NT2 * TILE_BYTES;
+constexpr int OFF_BARS = OFF_STAT + NT2 * STAT_BYTES;
+constexpr int OFF_MISC = OFF_BARS + NUM_BARS * 8;
+constexpr int SMEM_USED = OFF_MISC + 16;
+constexpr int SMEM_BYTES = 232448;   // the 227 KB a CTA may have; SMEM_USED plus the alignment gap must fit
 
 struct Params {
     const WorkItem *work;
@@ -78,8 +77,8 @@ struct Params {
     const int *cta_begin;
     int heads;
     long long stride_b, stride_h, stride_s;  // elements
-    const float *lse;     // [batch * heads, S], natural log
-    const float *delta;   // [batch * heads, S]
+    const float *lse2;    // [batch * heads * S] lse * log2 e
+    const float *delta;   // [batch * heads * S] rowsum(dO * O)
     __nv_bfloat16 *out_a; // DQ: dq; DKV: dk
     __nv_bfloat16 *out_b; // DKV: dv
     float scale, scale_log2;
@@ -88,32 +87,35 @@ struct Params {
     int *status;
 };
 
-__device__ __forceinline__ int sub_blocks(const WorkItem &it, int seg) {
-    return (it.seg_len[seg] + SUB - 1) / SUB;
+__device__ __forceinline__ int seg_blocks(const WorkItem &it, int seg) {
+    return (it.seg_len[seg] + BK - 1) / BK;
 }
 
-// acc = R T^T: resident tile (128 rows) times a streamed sub-block (64 rows), K = head dim.
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// acc = R T^T: resident tile (128 rows) times a streamed block (128 rows), K = head dim.
 __device__ __forceinline__ void issue_rt(uint32_t tmem_acc, uint32_t sR, uint32_t sT) {
-    constexpr uint32_t IDESC = idesc_bf16_f32(BM, SUB, 0, 0);
+    constexpr uint32_t IDESC = idesc_bf16_f32(BM, BK, 0, 0);
     const uint64_t da = smem_desc_sw128(sR, 16, 1024), db = smem_desc_sw128(sT, 16, 1024);
 #pragma unroll
     for (int k = 0; k < HD / 16; ++k) {
-        const uint64_t oa = (uint64_t)(((k >> 2) * RES_SLAB + (k & 3) * 32) >> 4);
-        const uint64_t ob = (uint64_t)(((k >> 2) * SUBT_SLAB + (k & 3) * 32) >> 4);
-        mma_ss(tmem_acc, da + oa, db + ob, IDESC, k > 0);
+        const uint64_t off = (uint64_t)(((k >> 2) * SLAB_BYTES + (k & 3) * 32) >> 4);
+        mma_ss(tmem_acc, da + off, db + off, IDESC, k > 0);
     }
 }
 
-// out (+)= A T: A (128 x 64, bf16) from TMEM, the streamed sub-block row-major in smem
-// (N-major operand: 64 rows of K, two 64-column slabs of N).
-// A sits where each element-wise warpgroup left it: the bf16 pairs of streamed rows
-// [32 w, 32 w + 32) occupy columns [32 w, 32 w + 16) of the fp32 block they were computed from.
-__device__ __forceinline__ void issue_at(uint32_t tmem_out, uint32_t tmem_a, uint32_t sT, bool accumulate) {
+// out (+)= A T: A (128 x 128, bf16) from TMEM, the streamed block row-major in smem (N-major
+// operand: 128 rows of K, two 64-column slabs of N).  The bf16 pairs of streamed rows
+// [32 g, 32 g + 32) sit 16 columns wide at column 32 g of region B (+ a_off).
+__device__ __forceinline__ void issue_at(uint32_t tmem_out, uint32_t tmem_b, uint32_t a_off, uint32_t sT,
+                                         bool accumulate) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
-    const uint64_t db = smem_desc_sw128(sT, SUBT_SLAB, 1024);
+    const uint64_t db = smem_desc_sw128(sT, SLAB_BYTES, 1024);
 #pragma unroll
-    for (int k = 0; k < SUB / 16; ++k)
-        mma_ts(tmem_out, tmem_a + (k >> 1) * 32 + (k & 1) * 8, db + (uint64_t)((k * 2048) >> 4), IDESC,
+    for (int k = 0; k < BK / 16; ++k)
+        mma_ts(tmem_out, tmem_b + (k >> 1) * 32 + a_off + (k & 1) * 8, db + (uint64_t)((k * 2048) >> 4), IDESC,
                (accumulate || k > 0) ? 1u : 0u);
 }
 
@@ -122,50 +124,63 @@ __global__ void __launch_bounds__(THREADS, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant__ CUtensorMap tmR2,
                 const __grid_constant__ CUtensorMap tmT1, const __grid_constant__ CUtensorMap tmT2,
                 const Params prm) {
-    constexpr int NST = nst_of(MODE);
-    constexpr int NB = nb_of(MODE), LA = NB - 1;          // MMAs run LA sub-blocks ahead of the element-wise step
-    constexpr uint32_t OUT_A = MODE == MODE_DKV ? 256 : 384, OUT_B = 384;  // TMEM columns of the outputs
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[NUM_BARS];
-    __shared__ uint32_t tmem_slot;
-    __shared__ int abort_flag;
-    __shared__ __align__(16) float stats[MODE == MODE_DKV ? NST : 1][2][SUB];  // DKV: lse (base 2), delta of streamed rows
+    constexpr uint32_t REG_A = 0, REG_B = 128, OUT_A = 256, OUT_B = 384;   // TMEM columns
 
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const uint32_t sR1 = smem_u32(smem), sR2 = sR1 + RES_BYTES;
-    const uint32_t sST = sR2 + RES_BYTES;
+    if ((int)(smem - smem_raw) + SMEM_USED > SMEM_BYTES) {
+        // the dynamic area starts too far from a 1024-byte boundary for everything to fit
+        if (threadIdx.x == 0 && atomicCAS(prm.status, 0, 0x900) == 0) prm.status[1] = blockIdx.x;
+        return;
+    }
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t sR1 = sbase + OFF_R1, sR2 = sbase + OFF_R2, sT1 = sbase + OFF_T1, sT2 = sbase + OFF_T2;
+    const float *stats = reinterpret_cast<const float *>(smem + OFF_STAT);
+    const uint32_t bar0 = sbase + OFF_BARS;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_MISC);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 4);
     const int tid = threadIdx.x, warp = tid >> 5;
-    const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     if (tid == 0) {
-        abort_flag = 0;
+        *abort_flag = 0;
         for (int i = 0; i < NUM_BARS; ++i) {
             uint32_t count = 1;
             if (i == EPI_DONE) count = 128;
-            if (i >= P_READY && i < P_READY + 3) count = 256;
+            if (i == A_DONE || i == P_READY) count = 256;
+            // DKV: ring 2 also carries the row statistics, copied by the 32 lanes of its producer warp
+            if (MODE == MODE_DKV && i >= T2_FULL && i < T2_FULL + NT2) count = 33;
             mbar_init(bar(i), count);
         }
         mbar_fence_init();
     }
     if (warp == 8) {
-        tmem_alloc(smem_u32(&tmem_slot), TMEM_COLS);
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = tmem_slot;
+    const uint32_t tmem = *tmem_slot;
     const int u_begin = prm.cta_begin[blockIdx.x], u_end = prm.cta_begin[blockIdx.x + 1];
 
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     }
-    if (warp == 8) {
-        // ------------------------------------------------ producer of the streamed sub-blocks
-        if (elect_one()) {
-            prefetch_tmap(&tmT1);
-            prefetch_tmap(&tmT2);
+    if (warp == 8 || warp == 10) {
+        // ------------------------------------------------ producers of the streamed blocks
+        // warp 8 feeds ring 1 (K_j in DQ mode, Q_i in DKV mode), warp 10 ring 2 (V_j / dO_i and,
+        // in DKV mode, the statistics of the streamed query rows)
+        const bool second = warp == 10;
+        const int lane = tid & 31;
+        const bool with_stats = MODE == MODE_DKV && second;   // whole warp takes part
+        const bool leader = with_stats ? lane == 0 : elect_one();
+        if (leader || with_stats) {
+            const CUtensorMap *tm = second ? &tmT2 : &tmT1;
+            if (leader) prefetch_tmap(tm);
+            const int nslot = second ? NT2 : NT1;
+            const int FULL = second ? T2_FULL : T1_FULL, EMPTY = second ? T2_EMPTY : T1_EMPTY;
+            const uint32_t ring = second ? sT2 : sT1;
             uint32_t g = 0;
             bool ok = true;
             for (int u = u_begin; ok && u < u_end; ++u) {
@@ -173,31 +188,49 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                 const WorkItem wi = prm.work[unit.item];
                 const int b = unit.bh / prm.heads, h = unit.bh % prm.heads;
                 for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
-                    const int nb = sub_blocks(wi, seg);
+                    const int nb = seg_blocks(wi, seg);
                     for (int j = 0; j < nb; ++j, ++g) {
-                        const int row = wi.seg_start[seg] + j * SUB;
-                        const uint32_t s = g % NST, ph = (g / NST) & 1;
-                        ok = wait_or_abort(bar(ST_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x402);
+                        const int row = wi.seg_start[seg] + j * BK;
+                        const uint32_t s = g % nslot, ph = (g / nslot) & 1;
+                        if (leader) ok = wait_or_abort(bar(EMPTY + s), ph ^ 1, abort_flag, prm.status, 0x402 + (second ? 1 : 0));
+                        if (with_stats) ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                         if (!ok) break;
-                        const uint32_t dst = sST + s * STAGE_BYTES;
-                        mbar_expect_tx(bar(ST_FULL + s), STAGE_BYTES);
-                        tma_load_4d(dst, &tmT1, bar(ST_FULL + s), 0, row, h, b);
-                        tma_load_4d(dst + SUBT_SLAB, &tmT1, bar(ST_FULL + s), 64, row, h, b);
-                        tma_load_4d(dst + SUBT_BYTES, &tmT2, bar(ST_FULL + s), 0, row, h, b);
-                        tma_load_4d(dst + SUBT_BYTES + SUBT_SLAB, &tmT2, bar(ST_FULL + s), 64, row, h, b);
+                        if (leader) {
+                            const uint32_t dst = ring + s * TILE_BYTES;
+                            mbar_expect_tx(bar(FULL + s), TILE_BYTES);
+                            tma_load_4d(dst, tm, bar(FULL + s), 0, row, h, b);
+                            tma_load_4d(dst + SLAB_BYTES, tm, bar(FULL + s), 64, row, h, b);
+                        }
+                        if (with_stats) {
+                            // lse2 and delta of the block's rows that lie inside the range (the others
+                            // are masked by position later); the arrival fires when the copies land
+                            const int valid = min(BK, wi.seg_len[seg] - j * BK);
+                            const long long p0 = (long long)unit.bh * prm.S + row;
+                            const uint32_t sdst = sbase + OFF_STAT + s * STAT_BYTES;
+#pragma unroll
+                            for (int i = 0; i < BK / 32; ++i) {
+                                const int c = lane + 32 * i;
+                                if (c < valid) {
+                                    cp_async4(sdst + 4 * c, prm.lse2 + p0 + c);
+                                    cp_async4(sdst + 4 * (BK + c), prm.delta + p0 + c);
+                                }
+                            }
+                            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar(FULL + s)) : "memory");
+                        }
                     }
                 }
             }
-            if (!ok) {
+            if (with_stats) asm volatile("cp.async.wait_all;" ::: "memory");
+            if (!ok && leader) {
                 // let every copy already issued land before the CTA retires
                 const long long t0 = clock64();
                 while (clock64() - t0 < 2000000) {
                 }
             }
         }
-    } else if (warp == 10) {
+    } else if (warp == 11) {
         // ------------------------------------------------ loader of the resident tiles
-        // A thread of its own, so that the sub-block producer can run ahead into the next unit
+        // A thread of its own, so that the block producers can run ahead into the next unit
         // while this one waits for the resident tiles to be released.
         if (elect_one()) {
             prefetch_tmap(&tmR1);
@@ -209,114 +242,28 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                 const WorkItem wi = prm.work[unit.item];
                 const int b = unit.bh / prm.heads, h = unit.bh % prm.heads;
                 // free once the last R T^T MMA of the previous unit has retired
-                if (uc > 0) ok = wait_or_abort(bar(RES_EMPTY), (uc - 1) & 1, &abort_flag, prm.status, 0x401);
+                if (uc > 0) ok = wait_or_abort(bar(RES_EMPTY), (uc - 1) & 1, abort_flag, prm.status, 0x401);
                 if (!ok) break;
-                mbar_expect_tx(bar(RES_FULL), 2 * RES_BYTES);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t off = (i >> 1) * RES_SLAB + (i & 1) * (SUB * 128);
-                    tma_load_4d(sR1 + off, &tmR1, bar(RES_FULL), (i >> 1) * 64, wi.q_start + (i & 1) * SUB, h, b);
-                    tma_load_4d(sR2 + off, &tmR2, bar(RES_FULL), (i >> 1) * 64, wi.q_start + (i & 1) * SUB, h, b);
-                }
+                mbar_expect_tx(bar(RES_FULL), 2 * TILE_BYTES);
+                tma_load_4d(sR1, &tmR1, bar(RES_FULL), 0, wi.q_start, h, b);
+                tma_load_4d(sR1 + SLAB_BYTES, &tmR1, bar(RES_FULL), 64, wi.q_start, h, b);
+                tma_load_4d(sR2, &tmR2, bar(RES_FULL), 0, wi.q_start, h, b);
+                tma_load_4d(sR2 + SLAB_BYTES, &tmR2, bar(RES_FULL), 64, wi.q_start, h, b);
                 if (u + 1 < u_end) {
                     // pull the next unit's resident tiles into L2 while this unit runs
                     const WorkUnit nu = prm.units[u + 1];
                     const int nq = prm.work[nu.item].q_start;
                     const int nb_ = nu.bh / prm.heads, nh = nu.bh % prm.heads;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        tma_prefetch_4d(&tmR1, (i >> 1) * 64, nq + (i & 1) * SUB, nh, nb_);
-                        tma_prefetch_4d(&tmR2, (i >> 1) * 64, nq + (i & 1) * SUB, nh, nb_);
-                    }
+                    tma_prefetch_4d(&tmR1, 0, nq, nh, nb_);
+                    tma_prefetch_4d(&tmR1, 64, nq, nh, nb_);
+                    tma_prefetch_4d(&tmR2, 0, nq, nh, nb_);
+                    tma_prefetch_4d(&tmR2, 64, nq, nh, nb_);
                 }
             }
             if (!ok) {
                 const long long t0 = clock64();
                 while (clock64() - t0 < 2000000) {
                 }
-            }
-        }
-    } else if (warp == 11) {
-        // ------------------------------------------------ DKV: statistics of the streamed query rows
-        // lse (base 2) and delta of the 64 rows of every sub-block go to shared memory, two
-        // sub-blocks ahead of use; rows beyond the range get lse = +inf, which turns their
-        // weights into exact zeros.
-        if (MODE == MODE_DKV) {
-            const int lane = tid & 31;
-            struct It {
-                int u, seg, j, bh;
-                WorkItem wi;
-                bool valid;
-            };
-            auto load_unit = [&](It &it) {
-                it.valid = it.u < u_end;
-                if (it.valid) {
-                    const WorkUnit unit = prm.units[it.u];
-                    it.wi = prm.work[unit.item];
-                    it.bh = unit.bh;
-                }
-            };
-            auto advance = [&](It &it) {
-                if (++it.j >= sub_blocks(it.wi, it.seg)) {
-                    it.j = 0;
-                    if (++it.seg >= it.wi.n_seg) {
-                        it.seg = 0;
-                        ++it.u;
-                        load_unit(it);
-                    }
-                }
-            };
-            auto fetch = [&](const It &it, float (&l2)[2], float (&dl)[2]) {
-                if (!it.valid) return;
-                const int row = it.wi.seg_start[it.seg] + it.j * SUB;
-                const int valid = min(SUB, it.wi.seg_len[it.seg] - it.j * SUB);
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int c = lane + 32 * i;
-                    l2[i] = __int_as_float(0x7f800000);
-                    dl[i] = 0.f;
-                    if (c < valid) {
-                        l2[i] = __ldg(prm.lse + (long long)it.bh * prm.S + row + c) * 1.4426950408889634f;
-                        dl[i] = __ldg(prm.delta + (long long)it.bh * prm.S + row + c);
-                    }
-                }
-            };
-            uint32_t g = 0;
-            bool ok = true;
-            auto publish = [&](const float (&l2)[2], const float (&dl)[2]) {
-                const uint32_t s = g % NST, ph = (g / NST) & 1;
-                if (lane == 0) ok = wait_or_abort(bar(ST_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x701);
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                if (!ok) return;
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    stats[s][0][lane + 32 * i] = l2[i];
-                    stats[s][1][lane + 32 * i] = dl[i];
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(STAT_FULL + s));
-                ++g;
-            };
-            It cur{u_begin, 0, 0, 0, WorkItem{}, false}, pre{u_begin, 0, 0, 0, WorkItem{}, false};
-            load_unit(cur);
-            load_unit(pre);
-            float al2[2], adl[2], bl2[2], bdl[2];
-            fetch(pre, al2, adl);
-            if (pre.valid) advance(pre);
-            fetch(pre, bl2, bdl);
-            if (pre.valid) advance(pre);
-            while (ok && cur.valid) {
-                publish(al2, adl);
-                if (!ok) break;
-                advance(cur);
-                fetch(pre, al2, adl);
-                if (pre.valid) advance(pre);
-                if (!cur.valid) break;
-                publish(bl2, bdl);
-                if (!ok) break;
-                advance(cur);
-                fetch(pre, bl2, bdl);
-                if (pre.valid) advance(pre);
             }
         }
     } else if (warp >= 12) {
@@ -331,7 +278,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
             const WorkItem wi = prm.work[unit.item];
             const int b = unit.bh / prm.heads, h = unit.bh % prm.heads;
             const bool row_ok = r < wi.q_rows;
-            ok = wait_or_abort(bar(OUT_FULL), uc & 1, &abort_flag, prm.status, 0x605);
+            ok = wait_or_abort(bar(OUT_FULL), uc & 1, abort_flag, prm.status, 0x605);
             if (!ok) break;
             tc_fence_after();
             const long long roff = (long long)b * prm.stride_b + (long long)h * prm.stride_h +
@@ -365,66 +312,62 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
     } else if (warp == 9) {
         // ---------------------------------------------------------- MMA issuer
         if (elect_one()) {
-            uint32_t g = 0, uc = 0;
-            uint32_t cP[3] = {0, 0, 0};
+            uint32_t g = 0, uc = 0;   // g: blocks issued so far (ring positions and barrier phases)
             bool ok = true;
-#ifdef HB_BWD_TIMING
-            long long tw_res = 0, tw_st = 0, tw_epi = 0, tw_p = 0, tw_st0 = 0, tw_p0 = 0, t_mark, t_start = clock64();
-#define TMARK() t_mark = clock64()
-#define TACC(x) x += clock64() - t_mark
-#else
-#define TMARK()
-#define TACC(x)
-#endif
+            auto t1 = [&](uint32_t e) { return sT1 + (e % NT1) * TILE_BYTES; };
+            auto t2 = [&](uint32_t e) { return sT2 + (e % NT2) * TILE_BYTES; };
             for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
                 const WorkItem wi = prm.work[prm.units[u].item];
-                const int n = wi.kv_blocks;  // sub-blocks of this item
-                TMARK();
-                ok = wait_or_abort(bar(RES_FULL), uc & 1, &abort_flag, prm.status, 0x501);
-                TACC(tw_res);
+                const int n = wi.kv_blocks;  // blocks of this item
+                ok = wait_or_abort(bar(RES_FULL), uc & 1, abort_flag, prm.status, 0x501);
                 if (!ok) break;
-                for (int s = 0; s < n + LA; ++s) {
-                    if (s < n) {
-                        const uint32_t e = g + s, slot = e % NST;
-                        TMARK();
-                        ok = wait_or_abort(bar(ST_FULL + slot), (e / NST) & 1, &abort_flag, prm.status, 0x502);
-                        TACC(tw_st);
-#ifdef HB_BWD_TIMING
-                        if (s < 2) tw_st0 += clock64() - t_mark;
-#endif
+                // scores and dP of the first block
+                ok = wait_or_abort(bar(T1_FULL + g % NT1), (g / NT1) & 1, abort_flag, prm.status, 0x502);
+                if (!ok) break;
+                tc_fence_after();
+                issue_rt(tmem + REG_A, sR1, t1(g));
+                mma_commit(bar(S_FULL));
+                ok = wait_or_abort(bar(T2_FULL + g % NT2), (g / NT2) & 1, abort_flag, prm.status, 0x503);
+                if (!ok) break;
+                tc_fence_after();
+                issue_rt(tmem + REG_B, sR2, t2(g));
+                mma_commit(bar(DP_FULL));
+                if (MODE == MODE_DQ) mma_commit(bar(T2_EMPTY + g % NT2));
+                if (n == 1) mma_commit(bar(RES_EMPTY));
+                for (int s = 0; s < n; ++s) {
+                    const uint32_t e = g + s;
+                    const bool more = s + 1 < n;
+                    if (more) {
+                        // scores of the next block, as soon as phase 1 has read this block's
+                        ok = wait_or_abort(bar(T1_FULL + (e + 1) % NT1), ((e + 1) / NT1) & 1, abort_flag, prm.status, 0x504);
+                        if (!ok) break;
+                        ok = wait_or_abort(bar(A_DONE), e & 1, abort_flag, prm.status, 0x505);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t sT = sST + slot * STAGE_BYTES;
-                        const uint32_t acc = tmem + (s % NB) * 128;
-                        issue_rt(acc, sR1, sT);
-                        issue_rt(acc + 64, sR2, sT + SUBT_BYTES);
-                        mma_commit(bar(S_FULL + (s % NB)));
-                        if (s == n - 1) mma_commit(bar(RES_EMPTY));
+                        issue_rt(tmem + REG_A, sR1, t1(e + 1));
+                        mma_commit(bar(S_FULL));
                     }
-                    if (s >= LA) {
-                        const int sp = s - LA, bf = sp % NB;
-                        const uint32_t e = g + sp, slot = e % NST;
-                        if (sp == 0 && uc > 0) {
-                            // the previous unit's accumulators have been read out
-                            TMARK();
-                            ok = wait_or_abort(bar(EPI_DONE), (uc - 1) & 1, &abort_flag, prm.status, 0x503);
-                            TACC(tw_epi);
-                            if (!ok) break;
-                        }
-                        TMARK();
-                        ok = wait_or_abort(bar(P_READY + bf), cP[bf] & 1, &abort_flag, prm.status, 0x504 + bf);
-                        TACC(tw_p);
-#ifdef HB_BWD_TIMING
-                        if (sp < 2) tw_p0 += clock64() - t_mark;
-#endif
+                    if (s == 0 && uc > 0) {
+                        // the previous unit's accumulators have been read out
+                        ok = wait_or_abort(bar(EPI_DONE), (uc - 1) & 1, abort_flag, prm.status, 0x506);
                         if (!ok) break;
-                        ++cP[bf];
+                    }
+                    ok = wait_or_abort(bar(P_READY), e & 1, abort_flag, prm.status, 0x507);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_at(tmem + OUT_A, tmem + REG_B, 16, t1(e), s > 0);                       // dS  x T1
+                    if (MODE == MODE_DKV) issue_at(tmem + OUT_B, tmem + REG_B, 0, t2(e), s > 0);   // P^T x T2
+                    mma_commit(bar(T1_EMPTY + e % NT1));
+                    if (MODE == MODE_DKV) mma_commit(bar(T2_EMPTY + e % NT2));
+                    if (more) {
+                        // dP of the next block overwrites P / dS of this one: after the MMAs above
+                        ok = wait_or_abort(bar(T2_FULL + (e + 1) % NT2), ((e + 1) / NT2) & 1, abort_flag, prm.status, 0x508);
+                        if (!ok) break;
                         tc_fence_after();
-                        const uint32_t sT = sST + slot * STAGE_BYTES;
-                        const uint32_t acc = tmem + bf * 128;
-                        issue_at(tmem + OUT_A, acc + 64, sT, sp > 0);                                  // dS  x T1
-                        if (MODE == MODE_DKV) issue_at(tmem + OUT_B, acc, sT + SUBT_BYTES, sp > 0);  // P^T x T2
-                        mma_commit(bar(ST_EMPTY + slot));
+                        issue_rt(tmem + REG_B, sR2, t2(e + 1));
+                        mma_commit(bar(DP_FULL));
+                        if (MODE == MODE_DQ) mma_commit(bar(T2_EMPTY + (e + 1) % NT2));
+                        if (s + 2 == n) mma_commit(bar(RES_EMPTY));   // last read of the resident tiles
                     }
                 }
                 if (!ok) break;
@@ -433,96 +376,132 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
             }
             // every MMA issued above has retired before TMEM is released
             mma_commit(bar(DRAIN));
-            wait_or_abort(bar(DRAIN), 0, &abort_flag, prm.status, 0x507);
-#ifdef HB_BWD_TIMING
-            atomicAdd(prm.status + 32 + MODE * 8 + 0, (int)(tw_res >> 6));
-            atomicAdd(prm.status + 32 + MODE * 8 + 1, (int)(tw_st >> 6));
-            atomicAdd(prm.status + 32 + MODE * 8 + 2, (int)(tw_epi >> 6));
-            atomicAdd(prm.status + 32 + MODE * 8 + 3, (int)(tw_p >> 6));
-            atomicAdd(prm.status + 32 + MODE * 8 + 4, (int)((clock64() - t_start) >> 6));
-            atomicMax(prm.status + 32 + MODE * 8 + 5, (int)((clock64() - t_start) >> 6));
-            atomicAdd(prm.status + 32 + MODE * 8 + 6, (int)(tw_st0 >> 6));
-            atomicAdd(prm.status + 32 + MODE * 8 + 7, (int)(tw_p0 >> 6));
-#endif
+            wait_or_abort(bar(DRAIN), 0, abort_flag, prm.status, 0x509);
         }
     } else if (warp < 8) {
-        // ------------------------------------ element-wise step + epilogue, warpgroup wg
+        // ------------------------------------ element-wise step, warpgroup wg: columns [64 wg, +64)
         asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
         const int wg = warp >> 2;
         const int r = tid & 127;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tA = tmem + lane_addr + REG_A + wg * 64, tB = tmem + lane_addr + REG_B + wg * 64;
         const float scale_log2 = prm.scale_log2;
-        uint32_t cS[3] = {0, 0, 0}, g = 0, uc = 0;
+        uint32_t g = 0;
         bool ok = true;
-        for (int u = u_begin; ok && u < u_end; ++u, ++uc) {
+        for (int u = u_begin; ok && u < u_end; ++u) {
             const WorkUnit unit = prm.units[u];
             const WorkItem wi = prm.work[unit.item];
             const int bh = unit.bh;
-            const int b = bh / prm.heads, h = bh % prm.heads;
-            const bool row_ok = r < wi.q_rows;
-            // DQ: this thread's query row statistics
+            // DQ: this thread's query row statistics; rows beyond the item get lse = +inf,
+            // which turns their weights into exact zeros
             float row_l2 = __int_as_float(0x7f800000), row_dl = 0.f;
-            if (MODE == MODE_DQ && row_ok) {
-                row_l2 = prm.lse[(long long)bh * prm.S + wi.q_start + r] * 1.4426950408889634f;
-                row_dl = prm.delta[(long long)bh * prm.S + wi.q_start + r];
+            if (MODE == MODE_DQ && r < wi.q_rows) {
+                row_l2 = __ldg(prm.lse2 + (long long)bh * prm.S + wi.q_start + r);
+                row_dl = __ldg(prm.delta + (long long)bh * prm.S + wi.q_start + r);
             }
-            int s = 0;
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
-                const int nb = sub_blocks(wi, seg);
-                for (int j = 0; j < nb; ++j, ++s) {
-                    const int bf = s % NB;
-                    // this warpgroup's 32 columns of the sub-block
-                    const int valid = min(SUB, wi.seg_len[seg] - j * SUB) - wg * 32;
-                    const uint32_t tAcc = tmem + lane_addr + bf * 128;
-                    const uint32_t e = g + s, slot = e % NST;
+                const int nb = seg_blocks(wi, seg);
+                for (int j = 0; j < nb; ++j, ++g) {
+                    // streamed rows of this warpgroup that lie inside the range
+                    const int valid = min(BK, wi.seg_len[seg] - j * BK) - wg * 64;
+                    const float4 *st_l = nullptr, *st_d = nullptr;
                     if (MODE == MODE_DKV) {
-                        ok = wait_or_abort(bar(STAT_FULL + slot), (e / NST) & 1, &abort_flag, prm.status, 0x601 + wg);
+                        // the statistics arrive with ring 2
+                        ok = wait_or_abort(bar(T2_FULL + g % NT2), (g / NT2) & 1, abort_flag, prm.status, 0x601 + wg);
                         if (!ok) break;
+                        st_l = reinterpret_cast<const float4 *>(stats + (g % NT2) * (2 * BK) + wg * 64);
+                        st_d = st_l + BK / 4;
                     }
-                    ok = wait_or_abort(bar(S_FULL + bf), cS[bf] & 1, &abort_flag, prm.status, 0x603 + wg);
+                    // ---- phase 1: weights from the scores
+                    ok = wait_or_abort(bar(S_FULL), g & 1, abort_flag, prm.status, 0x603 + wg);
                     if (!ok) break;
                     tc_fence_after();
-                    uint32_t a1[32], a2[32];
-                    tmem_ld32(tAcc + wg * 32, a1);
-                    tmem_ld32(tAcc + 64 + wg * 32, a2);
+                    uint32_t a[64];
+                    tmem_ld32(tA, *reinterpret_cast<uint32_t(*)[32]>(&a[0]));
+                    tmem_ld32(tA + 32, *reinterpret_cast<uint32_t(*)[32]>(&a[32]));
                     tmem_wait_ld();
-                    uint32_t pk[16], dk[16];
+                    tc_fence_before();
+                    mbar_arrive(bar(A_DONE));   // region A may take the next block's scores
+                    const bool ragged = valid < 64;   // only the last block of a range
+                    auto phase1 = [&](auto RAGGED) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int c0 = 2 * i;
-                        float l0, l1, d0, d1;
-                        if (MODE == MODE_DKV) {
-                            const float2 l2 = *reinterpret_cast<const float2 *>(&stats[slot][0][wg * 32 + c0]);
-                            const float2 dl = *reinterpret_cast<const float2 *>(&stats[slot][1][wg * 32 + c0]);
-                            l0 = l2.x; l1 = l2.y; d0 = dl.x; d1 = dl.y;
-                        } else {
-                            l0 = l1 = row_l2;
-                            d0 = d1 = row_dl;
+                        for (int c4 = 0; c4 < 16; ++c4) {
+                            float4 l4 = make_float4(row_l2, row_l2, row_l2, row_l2);
+                            if (MODE == MODE_DKV) l4 = st_l[c4];
+                            const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(a[4 * c4]), __uint_as_float(a[4 * c4 + 1])),
+                                                         make_float2(scale_log2, scale_log2), make_float2(-l4.x, -l4.y));
+                            const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(a[4 * c4 + 2]), __uint_as_float(a[4 * c4 + 3])),
+                                                         make_float2(scale_log2, scale_log2), make_float2(-l4.z, -l4.w));
+                            // (a polynomial exp2 on the FMA pipes for part of the pairs, as in the forward
+                            // kernel, measured equal here: this step is not bound by the MUFU unit)
+                            float2 p0, p1;
+                            p0.x = ex2(x0.x);
+                            p0.y = ex2(x0.y);
+                            p1.x = ex2(x1.x);
+                            p1.y = ex2(x1.y);
+                            if (decltype(RAGGED)::value) {
+                                // rows beyond the end of the range (their statistics are stale)
+                                if (4 * c4 >= valid) p0.x = 0.f;
+                                if (4 * c4 + 1 >= valid) p0.y = 0.f;
+                                if (4 * c4 + 2 >= valid) p1.x = 0.f;
+                                if (4 * c4 + 3 >= valid) p1.y = 0.f;
+                            }
+                            a[4 * c4] = __float_as_uint(p0.x);
+                            a[4 * c4 + 1] = __float_as_uint(p0.y);
+                            a[4 * c4 + 2] = __float_as_uint(p1.x);
+                            a[4 * c4 + 3] = __float_as_uint(p1.y);
                         }
-                        float p0 = ex2(fmaf(__uint_as_float(a1[c0]), scale_log2, -l0));
-                        float p1 = ex2(fmaf(__uint_as_float(a1[c0 + 1]), scale_log2, -l1));
-                        if (MODE == MODE_DQ) {
-                            // keys beyond the end of the range
-                            if (c0 >= valid) p0 = 0.f;
-                            if (c0 + 1 >= valid) p1 = 0.f;
+                    };
+                    if (ragged) phase1(std::true_type{});
+                    else phase1(std::false_type{});
+                    // ---- phase 2: dS = P * (dP - delta), written over dP together with P
+                    ok = wait_or_abort(bar(DP_FULL), g & 1, abort_flag, prm.status, 0x605 + wg);
+                    if (!ok) break;
+                    tc_fence_after();
+                    auto phase2 = [&](auto RAGGED) {
+#pragma unroll
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            uint32_t d[32];
+                            tmem_ld32(tB + h2 * 32, d);
+                            tmem_wait_ld();
+                            uint32_t pk[16], dk[16];
+#pragma unroll
+                            for (int i4 = 0; i4 < 8; ++i4) {
+                                const int c0 = h2 * 32 + 4 * i4;
+                                float4 d4 = make_float4(row_dl, row_dl, row_dl, row_dl);
+                                if (MODE == MODE_DKV) d4 = st_d[c0 >> 2];
+                                const float2 pa = make_float2(__uint_as_float(a[c0]), __uint_as_float(a[c0 + 1]));
+                                const float2 pb = make_float2(__uint_as_float(a[c0 + 2]), __uint_as_float(a[c0 + 3]));
+                                float2 sa = __fadd2_rn(make_float2(__uint_as_float(d[4 * i4]), __uint_as_float(d[4 * i4 + 1])),
+                                                       make_float2(-d4.x, -d4.y));
+                                float2 sb = __fadd2_rn(make_float2(__uint_as_float(d[4 * i4 + 2]), __uint_as_float(d[4 * i4 + 3])),
+                                                       make_float2(-d4.z, -d4.w));
+                                sa = __fmul2_rn(sa, pa);
+                                sb = __fmul2_rn(sb, pb);
+                                if (decltype(RAGGED)::value) {
+                                    // P is zero there already; dP - delta may be anything
+                                    if (c0 >= valid) sa.x = 0.f;
+                                    if (c0 + 1 >= valid) sa.y = 0.f;
+                                    if (c0 + 2 >= valid) sb.x = 0.f;
+                                    if (c0 + 3 >= valid) sb.y = 0.f;
+                                }
+                                pk[2 * i4] = pack_bf16(pa.x, pa.y);
+                                pk[2 * i4 + 1] = pack_bf16(pb.x, pb.y);
+                                dk[2 * i4] = pack_bf16(sa.x, sa.y);
+                                dk[2 * i4 + 1] = pack_bf16(sb.x, sb.y);
+                            }
+                            // the 32 columns just read take P (16 columns of bf16 pairs) and dS (16)
+                            if (MODE == MODE_DKV) tmem_st16(tB + h2 * 32, pk);
+                            tmem_st16(tB + h2 * 32 + 16, dk);
                         }
-                        const float s0 = p0 * (__uint_as_float(a2[c0]) - d0);
-                        const float s1 = p1 * (__uint_as_float(a2[c0 + 1]) - d1);
-                        pk[i] = pack_bf16(p0, p1);
-                        dk[i] = pack_bf16(s0, s1);
-                    }
-                    // in place: the bf16 pairs land in the first half of the 32 fp32 columns this
-                    // warpgroup has just read, so no other thread's data is touched
-                    if (MODE == MODE_DKV) tmem_st16(tAcc + wg * 32, pk);
-                    tmem_st16(tAcc + 64 + wg * 32, dk);
-                    ++cS[bf];
+                    };
+                    if (ragged) phase2(std::true_type{});
+                    else phase2(std::false_type{});
                     tmem_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar(P_READY + bf));
+                    mbar_arrive(bar(P_READY));
                 }
             }
-            if (!ok) break;
-            g += wi.kv_blocks;
         }
     }
 
@@ -534,10 +513,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
     }
 }
 
-// delta[bh, r] = sum_d dO[r, d] * O[r, d]: one warp per row, 8 bytes per lane.
+// lse2[row] = lse[row] * log2 e, delta[row] = sum_d dO[row, d] * O[row, d]: one warp per row, 8 bytes per lane.
 __global__ void __launch_bounds__(256)
-delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__restrict__ out, float *__restrict__ delta,
-             int S, int heads, long long stride_b, long long stride_h, long long stride_s, long long n_rows) {
+delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__restrict__ out,
+             const float *__restrict__ lse, float *__restrict__ lse2, float *__restrict__ delta, int S, int heads,
+             long long stride_b, long long stride_h, long long stride_s, long long n_rows) {
     const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= n_rows) return;
     const int lane = threadIdx.x & 31;
@@ -553,7 +533,10 @@ delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__rest
     float acc = a0.x * c0.x + a0.y * c0.y + a1.x * c1.x + a1.y * c1.y;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) delta[row] = acc;
+    if (lane == 0) {
+        lse2[row] = lse[row] * 1.4426950408889634f;
+        delta[row] = acc;
+    }
 }
 
 void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, const int *seg_start,
@@ -568,7 +551,7 @@ void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, cons
             if (seg_len[s] <= 0) continue;
             it.seg_start[it.n_seg] = seg_start[s];
             it.seg_len[it.n_seg] = seg_len[s];
-            it.kv_blocks += (seg_len[s] + SUB - 1) / SUB;
+            it.kv_blocks += (seg_len[s] + BK - 1) / BK;
             ++it.n_seg;
         }
         items.push_back(it);
@@ -578,8 +561,8 @@ void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, cons
 }  // namespace
 
 // Work list of the backward kernels: 128 resident rows per item, the rows they exchange
-// gradients with listed as up to three contiguous ranges and counted in sub-blocks of 64.
-// Also allocates the delta scratch.  Called from hilberta_plan_bind for bf16 bindings.
+// gradients with listed as up to three contiguous ranges and counted in blocks of 128.
+// Also allocates the per-row scratch: lse * log2 e for every row, then delta for every row.  Called from hilberta_plan_bind for bf16 bindings.
 int attn_bwd_prepare(hilberta_plan_t *p) {
     std::vector<WorkItem> items;
     {
@@ -638,14 +621,14 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
     HB_CUDA(cudaMemcpy(p->d_bwd_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
     HB_CUDA(cudaMalloc(&p->d_bwd_cta_begin, sizeof(int) * cta_begin.size()));
     HB_CUDA(cudaMemcpy(p->d_bwd_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
-    HB_CUDA(cudaMalloc(&p->d_delta, sizeof(float) * (size_t)bh * p->S));
+    HB_CUDA(cudaMalloc(&p->d_delta, sizeof(float) * 2 * (size_t)bh * p->S));
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes_of(MODE_DQ));
+        attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            smem_bytes_of(MODE_DKV));
+                                            SMEM_BYTES);
     });
     HB_CUDA(attr_err);
     return HILBERTA_OK;
@@ -657,14 +640,14 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
     if (p->n_bwd_work == 0) return HILBERTA_OK;
     CUtensorMap mq, mk, mv, mdo;
     int rc;
-    if ((rc = make_tensor_map(&mq, q, p, SUB)) != HILBERTA_OK) return rc;
-    if ((rc = make_tensor_map(&mk, k, p, SUB)) != HILBERTA_OK) return rc;
-    if ((rc = make_tensor_map(&mv, v, p, SUB)) != HILBERTA_OK) return rc;
-    if ((rc = make_tensor_map(&mdo, dout, p, SUB)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mq, q, p, BK)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mk, k, p, BK)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mv, v, p, BK)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mdo, dout, p, BK)) != HILBERTA_OK) return rc;
     const long long n_rows = (long long)p->batch * p->heads * p->S;
     delta_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, stream>>>(
-        (const __nv_bfloat16 *)dout, (const __nv_bfloat16 *)out, delta, p->S, p->heads, p->stride_b, p->stride_h,
-        p->stride_s, n_rows);
+        (const __nv_bfloat16 *)dout, (const __nv_bfloat16 *)out, lse, delta, delta + n_rows, p->S, p->heads,
+        p->stride_b, p->stride_h, p->stride_s, n_rows);
     HB_LAUNCHED();
     Params prm;
     prm.work = p->d_bwd_work;
@@ -674,8 +657,8 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
     prm.stride_b = p->stride_b;
     prm.stride_h = p->stride_h;
     prm.stride_s = p->stride_s;
-    prm.lse = lse;
-    prm.delta = delta;
+    prm.lse2 = delta;
+    prm.delta = delta + n_rows;
     prm.scale = p->scale;
     prm.scale_log2 = p->scale * 1.4426950408889634f;
     prm.S = p->S;
@@ -684,11 +667,11 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
                        ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
     prm.out_a = (__nv_bfloat16 *)dq;
     prm.out_b = nullptr;
-    attn_bwd_kernel<MODE_DQ><<<p->n_bwd_cta, THREADS, smem_bytes_of(MODE_DQ), stream>>>(mq, mdo, mk, mv, prm);
+    attn_bwd_kernel<MODE_DQ><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mq, mdo, mk, mv, prm);
     HB_LAUNCHED();
     prm.out_a = (__nv_bfloat16 *)dk;
     prm.out_b = (__nv_bfloat16 *)dv;
-    attn_bwd_kernel<MODE_DKV><<<p->n_bwd_cta, THREADS, smem_bytes_of(MODE_DKV), stream>>>(mk, mv, mq, mdo, prm);
+    attn_bwd_kernel<MODE_DKV><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mk, mv, mq, mdo, prm);
     HB_LAUNCHED();
     return HILBERTA_OK;
 }
@@ -744,8 +727,8 @@ extern "C" int hilberta_backward_static(const void *dout, const void *q, const v
     }
     for (int j = 0; j < 5; ++j) bits |= (uintptr_t)in[j];
     if (bits & 15) return HILBERTA_ERR_INVALID;
-    // one float of scratch per (batch, head, token): refuse what the fixed array cannot hold
-    if ((unsigned long long)p->batch * p->heads * p->S > (unsigned long long)HILBERTA_STATIC_SCRATCH_FLOATS)
+    // two floats of scratch per (batch, head, token): refuse what the fixed array cannot hold
+    if (2ull * p->batch * p->heads * p->S > (unsigned long long)HILBERTA_STATIC_SCRATCH_FLOATS)
         return HILBERTA_ERR_BUFFER;
     int dev = -1;
     HB_CUDA(cudaGetDevice(&dev));
