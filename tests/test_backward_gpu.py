@@ -155,3 +155,35 @@ def test_backward_flux2048_sampled():
             gsel = gt[:, h:h + 1][:, :, toks].double().numpy()
             assert orc.rel_l2_err(gsel, r) <= 5e-3, (name, h, orc.rel_l2_err(gsel, r))
             assert orc.max_abs_err(gsel, r) <= 1e-2 * max(1.0, np.abs(r).max()), (name, h)
+
+
+def test_backward_strided_tensors():
+    """All eight tensors as views with the same non-dense strides (heads interleaved per token)."""
+    H = W = 16
+    nt, heads, B = 24, 3, 2
+    S = nt + H * W
+    g = torch.Generator().manual_seed(31)
+    packs = [torch.randn((B, S, heads, 128), generator=g).to(torch.bfloat16).cuda() for _ in range(4)]
+    q, k, v, do = (t.permute(0, 2, 1, 3) for t in packs)          # [B, heads, S, D] views, stride_s = heads * D
+    plan = hb.Plan(H, W, 64, 16, 2, nt)
+    try:
+        plan.bind_like(q)
+        view = lambda: torch.empty((B, S, heads, 128), device="cuda", dtype=torch.bfloat16).permute(0, 2, 1, 3)
+        out, dq, dk, dv = view(), view(), view(), view()
+        lse = torch.empty((B, heads, S), device="cuda", dtype=torch.float32)
+        plan.forward_lse(q, k, v, out, lse)
+        plan.backward(do, q, k, v, out, lse, dq, dk, dv)
+        assert plan.status() == 0
+        # the same problem on dense copies
+        qc, kc, vc, doc = (t.contiguous() for t in (q, k, v, do))
+        plan.bind_like(qc)
+        outc, dqc, dkc, dvc = (torch.empty_like(qc) for _ in range(4))
+        lsec = torch.empty_like(lse)
+        plan.forward_lse(qc, kc, vc, outc, lsec)
+        plan.backward(doc, qc, kc, vc, outc, lsec, dqc, dkc, dvc)
+        assert plan.status() == 0
+        for a, b in ((out, outc), (dq, dqc), (dk, dkc), (dv, dvc)):
+            assert torch.equal(a.contiguous().view(torch.int16), b.view(torch.int16))
+        assert torch.equal(lse, lsec)
+    finally:
+        plan.destroy()
