@@ -340,7 +340,7 @@ def main():
             e2e_ms = float(t.item())
         e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": 3 * tensor_bytes, "d2h_bytes_per_step": tensor_bytes,
-               "api": "hilberta_forward_host (pinned host buffers; H2D, one launch with entry and exit gathers fused in, D2H)",
+               "api": "hilberta_forward_host (pinned host buffers; per slice of heads: H2D, one launch with entry and exit gathers fused in, D2H; the slices are pipelined over two copy streams)",
                "steps": n_e2e}
         assert torch.isfinite(oh.float()).all()
 

@@ -652,10 +652,11 @@ EncodeTiledFn encode_fn() {
 }  // namespace
 
 // [batch, heads, S, 128] bf16 with element strides -> 4-D map, box = 64 columns x box_rows rows.
-int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, int box_rows) {
+int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, int box_rows, int heads) {
+    if (heads <= 0) heads = p->heads;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return HILBERTA_ERR_CUDA;
-    cuuint64_t dims[4] = {128, (cuuint64_t)p->S, (cuuint64_t)p->heads, (cuuint64_t)p->batch};
+    cuuint64_t dims[4] = {128, (cuuint64_t)p->S, (cuuint64_t)heads, (cuuint64_t)p->batch};
     cuuint64_t strides[3] = {(cuuint64_t)p->stride_s * 2, (cuuint64_t)p->stride_h * 2, (cuuint64_t)p->stride_b * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -698,6 +699,42 @@ int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
     return HILBERTA_OK;
 }
 
+// Static schedule: every (item, batch*head) unit goes to the least-loaded CTA, longest units
+// first (cost = MMA block pairs + a fixed per-unit overhead); units are stored grouped by CTA.
+static int upload_schedule(const std::vector<WorkItem> &items, int bh, int sm_count, WorkUnit **d_units,
+                           int **d_cta_begin, int *n_cta_out) {
+    const long long n_units = (long long)items.size() * bh;
+    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    const int n_cta = (int)std::min<long long>(n_units, sm_count);
+    std::vector<std::vector<WorkUnit>> bins(n_cta);
+    typedef std::pair<long long, int> Load;  // (load, cta)
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
+    for (int i = 0; i < (int)items.size(); ++i) {
+        const long long cost = (long long)items[i].kv_blocks * (items[i].q_rows > BM ? 2 : 1) + 2;
+        for (int j = 0; j < bh; ++j) {
+            Load top = heap.top();
+            heap.pop();
+            bins[top.second].push_back(WorkUnit{i, j});
+            heap.push(Load(top.first + cost, top.second));
+        }
+    }
+    std::vector<WorkUnit> units;
+    std::vector<int> cta_begin(n_cta + 1, 0);
+    units.reserve((size_t)n_units);
+    for (int c = 0; c < n_cta; ++c) {
+        cta_begin[c] = (int)units.size();
+        units.insert(units.end(), bins[c].begin(), bins[c].end());
+    }
+    cta_begin[n_cta] = (int)units.size();
+    *n_cta_out = n_cta;
+    HB_CUDA(cudaMalloc(d_units, sizeof(WorkUnit) * units.size()));
+    HB_CUDA(cudaMemcpy(*d_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
+    HB_CUDA(cudaMalloc(d_cta_begin, sizeof(int) * cta_begin.size()));
+    HB_CUDA(cudaMemcpy(*d_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
+    return HILBERTA_OK;
+}
+
 // Work list: prefix rows read the whole sequence; the rows of each slid tile
 // read the prefix and the tile's own one or two ranges.  Longest items first.
 int attn_bf16_prepare(hilberta_plan_t *p) {
@@ -720,47 +757,34 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
     cudaFree(p->d_work);
     cudaFree(p->d_units);
     cudaFree(p->d_cta_begin);
+    cudaFree(p->d_units_chunk);
+    cudaFree(p->d_cta_begin_chunk);
     p->d_work = nullptr;
     p->d_units = nullptr;
     p->d_cta_begin = nullptr;
+    p->d_units_chunk = nullptr;
+    p->d_cta_begin_chunk = nullptr;
+    p->n_cta_chunk = 0;
     p->n_work = (int)items.size();
     p->n_cta = 0;
     if (items.empty()) return HILBERTA_OK;
 
-    // Static schedule: every (item, batch*head) unit goes to the least-loaded CTA,
-    // longest units first.  Cost = MMA block pairs + a fixed per-unit overhead.
-    const int bh = p->batch * p->heads;
-    const long long n_units = (long long)items.size() * bh;
-    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
-    const int n_cta = (int)std::min<long long>(n_units, p->sm_count);
-    std::vector<std::vector<WorkUnit>> bins(n_cta);
-    typedef std::pair<long long, int> Load;  // (load, cta)
-    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
-    for (int i = 0; i < (int)items.size(); ++i) {
-        const long long cost = (long long)items[i].kv_blocks * (items[i].q_rows > BM ? 2 : 1) + 2;
-        for (int j = 0; j < bh; ++j) {
-            Load top = heap.top();
-            heap.pop();
-            bins[top.second].push_back(WorkUnit{i, j});
-            heap.push(Load(top.first + cost, top.second));
-        }
-    }
-    std::vector<WorkUnit> units;
-    std::vector<int> cta_begin(n_cta + 1, 0);
-    units.reserve((size_t)n_units);
-    for (int c = 0; c < n_cta; ++c) {
-        cta_begin[c] = (int)units.size();
-        units.insert(units.end(), bins[c].begin(), bins[c].end());
-    }
-    cta_begin[n_cta] = (int)units.size();
-    p->n_cta = n_cta;
     HB_CUDA(cudaMalloc(&p->d_work, sizeof(WorkItem) * items.size()));
     HB_CUDA(cudaMemcpy(p->d_work, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
-    HB_CUDA(cudaMalloc(&p->d_units, sizeof(WorkUnit) * units.size()));
-    HB_CUDA(cudaMemcpy(p->d_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
-    HB_CUDA(cudaMalloc(&p->d_cta_begin, sizeof(int) * cta_begin.size()));
-    HB_CUDA(cudaMemcpy(p->d_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
+    int rc = upload_schedule(items, p->batch * p->heads, p->sm_count, &p->d_units, &p->d_cta_begin, &p->n_cta);
+    if (rc != HILBERTA_OK) return rc;
+    // slice of heads for the pipelined host-buffer path: the divisor of `heads` nearest to a quarter
+    p->chunk_heads = p->heads;
+    for (int d = (p->heads + 3) / 4; d >= 1; --d)
+        if (p->heads % d == 0) {
+            p->chunk_heads = d;
+            break;
+        }
+    if (p->chunk_heads < p->heads) {
+        rc = upload_schedule(items, p->batch * p->chunk_heads, p->sm_count, &p->d_units_chunk, &p->d_cta_begin_chunk,
+                             &p->n_cta_chunk);
+        if (rc != HILBERTA_OK) return rc;
+    }
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
@@ -774,18 +798,34 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
 }
 
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream) {
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk) {
     if (p->n_work == 0) return HILBERTA_OK;
+    int heads = p->heads, n_cta = p->n_cta;
+    const WorkUnit *units = p->d_units;
+    const int *cta_begin = p->d_cta_begin;
+    if (chunk >= 0 && p->chunk_heads < p->heads) {
+        // a slice of heads: same strides, shifted base pointers, the slice's own schedule
+        if (lse) return HILBERTA_ERR_INVALID;
+        heads = p->chunk_heads;
+        const long long off = (long long)chunk * heads * p->stride_h;
+        q = (const __nv_bfloat16 *)q + off;
+        k = (const __nv_bfloat16 *)k + off;
+        v = (const __nv_bfloat16 *)v + off;
+        out = (__nv_bfloat16 *)out + off;
+        units = p->d_units_chunk;
+        cta_begin = p->d_cta_begin_chunk;
+        n_cta = p->n_cta_chunk;
+    }
     CUtensorMap mq, mk, mv;
     int rc;
-    if ((rc = make_tensor_map(&mq, q, p, BN)) != HILBERTA_OK) return rc;
-    if ((rc = make_tensor_map(&mk, k, p, BN)) != HILBERTA_OK) return rc;
-    if ((rc = make_tensor_map(&mv, v, p, BN)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mq, q, p, BN, heads)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mk, k, p, BN, heads)) != HILBERTA_OK) return rc;
+    if ((rc = make_tensor_map(&mv, v, p, BN, heads)) != HILBERTA_OK) return rc;
     Params prm;
     prm.work = p->d_work;
-    prm.units = p->d_units;
-    prm.cta_begin = p->d_cta_begin;
-    prm.heads = p->heads;
+    prm.units = units;
+    prm.cta_begin = cta_begin;
+    prm.heads = heads;
     prm.stride_b = p->stride_b;
     prm.stride_h = p->stride_h;
     prm.stride_s = p->stride_s;
@@ -803,11 +843,11 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
         gprm.gq = (const __nv_bfloat16 *)q;
         gprm.gk = (const __nv_bfloat16 *)k;
         gprm.gv = (const __nv_bfloat16 *)v;
-        attn_bf16_kernel<true><<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, gprm);
+        attn_bf16_kernel<true><<<n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, gprm);
     } else {
         KernelParams<false> pprm;
         static_cast<Params &>(pprm) = prm;
-        attn_bf16_kernel<false><<<p->n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, pprm);
+        attn_bf16_kernel<false><<<n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, pprm);
     }
     HB_LAUNCHED();
     return HILBERTA_OK;

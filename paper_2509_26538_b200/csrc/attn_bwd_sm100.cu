@@ -36,7 +36,7 @@
 namespace hilberta {
 using namespace ptx;
 
-int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, int box_rows);
+int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, int box_rows, int heads = 0);
 
 namespace {
 

@@ -113,16 +113,27 @@ attn_fp32_kernel(const float *__restrict__ q, const float *__restrict__ k, const
 }
 
 int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream) {
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk) {
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
     if ((bits & 15) || ((p->stride_b | p->stride_h | p->stride_s) & 3)) return HILBERTA_ERR_INVALID;
-    dim3 grid((p->S + kRowsPerBlock - 1) / kRowsPerBlock, p->batch * p->heads);
+    int heads = p->heads;
+    if (chunk >= 0) {
+        // a slice of heads: same strides, shifted base pointers
+        if (lse) return HILBERTA_ERR_INVALID;
+        heads = p->chunk_heads;
+        const long long off = (long long)chunk * heads * p->stride_h;
+        q = (const float *)q + off;
+        k = (const float *)k + off;
+        v = (const float *)v + off;
+        out = (float *)out + off;
+    }
+    dim3 grid((p->S + kRowsPerBlock - 1) / kRowsPerBlock, p->batch * heads);
     dim3 block(kRowsPerBlock * 32);
 #define HB_FP32_CASE(DD)                                                                              \
     case DD:                                                                                          \
         attn_fp32_kernel<DD><<<grid, block, 0, stream>>>(                                             \
             (const float *)q, (const float *)k, (const float *)v, (float *)out, p->stride_b,          \
-            p->stride_h, p->stride_s, p->heads, p->S, p->P, p->d_row_window, p->d_windows, out_map, in_map,   \
+            p->stride_h, p->stride_s, heads, p->S, p->P, p->d_row_window, p->d_windows, out_map, in_map,   \
             lse, p->scale);                                                                                \
         break;
     switch (p->head_dim) {

@@ -85,6 +85,14 @@ struct hilberta_plan_s {
     hilberta::WorkUnit *d_units;  // [n_work * batch * heads], grouped by CTA
     int *d_cta_begin;             // [n_cta + 1]
     int n_cta;
+    // a second schedule over a slice of chunk_heads heads (all batches), for the host-buffer entry
+    // point, which pipelines copies and launches slice by slice; chunk_heads == heads: no slicing
+    int chunk_heads;
+    hilberta::WorkUnit *d_units_chunk;
+    int *d_cta_begin_chunk;
+    int n_cta_chunk;
+    cudaStream_t s_in, s_out;           // copy streams of hilberta_forward_host (created on first use)
+    std::vector<cudaEvent_t> ev_in, ev_done;
     // backward pass: 128-row items over the same key lists, their schedule, and the
     // per-row scratch delta = rowsum(dO * O) that both backward kernels read
     hilberta::WorkItem *d_bwd_work;
@@ -107,10 +115,12 @@ namespace hilberta {
 // (natural log), indexed like `out` rows.
 // in_map: nullptr = q, k, v are in physical order; else they are in ORIGINAL order and physical
 // row p is read from row in_map[p] (the entry gather fused into the loads).
+// chunk: -1 = the whole bound problem; c >= 0 = heads [c * chunk_heads, (c + 1) * chunk_heads) of
+// every batch item only (lse must be null then).
 int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream);
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk = -1);
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
-                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream);
+                     float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk = -1);
 int attn_bf16_prepare(hilberta_plan_t *p);
 int attn_bwd_prepare(hilberta_plan_t *p);
 // dq, dk, dv (bf16, physical order, the bound strides) from dout, q, k, v, out and the forward's lse.

@@ -263,6 +263,12 @@ static void free_plan(hilberta_plan_t *p) {
     cudaFree(p->d_work);
     cudaFree(p->d_units);
     cudaFree(p->d_cta_begin);
+    cudaFree(p->d_units_chunk);
+    cudaFree(p->d_cta_begin_chunk);
+    for (cudaEvent_t e : p->ev_in) cudaEventDestroy(e);
+    for (cudaEvent_t e : p->ev_done) cudaEventDestroy(e);
+    if (p->s_in) cudaStreamDestroy(p->s_in);
+    if (p->s_out) cudaStreamDestroy(p->s_out);
     cudaFree(p->d_bwd_work);
     cudaFree(p->d_bwd_units);
     cudaFree(p->d_bwd_cta_begin);
@@ -561,7 +567,8 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
 }
 
 static int forward_impl(const void *q, const void *k, const void *v, void *out, float *lse,
-                        const hilberta_plan_t *p, const int *out_map, const int *in_map, void *stream) {
+                        const hilberta_plan_t *p, const int *out_map, const int *in_map, void *stream,
+                        int chunk = -1) {
     if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
     if (out == q || out == k || out == v) return HILBERTA_ERR_INVALID;
@@ -569,10 +576,10 @@ static int forward_impl(const void *q, const void *k, const void *v, void *out, 
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;  // the plan's tables live on another device
     cudaStream_t st = (cudaStream_t)stream;
-    if (p->dtype == HILBERTA_FP32) return launch_attn_fp32(p, q, k, v, out, lse, out_map, in_map, st);
+    if (p->dtype == HILBERTA_FP32) return launch_attn_fp32(p, q, k, v, out, lse, out_map, in_map, st, chunk);
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
     if (bits & 15) return HILBERTA_ERR_INVALID;
-    return launch_attn_bf16(p, q, k, v, out, lse, out_map, in_map, st);
+    return launch_attn_bf16(p, q, k, v, out, lse, out_map, in_map, st, chunk);
 }
 
 extern "C" int hilberta_forward(const void *q, const void *k, const void *v, void *out,
@@ -621,9 +628,11 @@ extern "C" int hilberta_backward(const void *dout, const void *q, const void *k,
     return launch_attn_bwd(p, dout, q, k, v, out, lse, dq, dk, dv, p->d_delta, (cudaStream_t)stream);
 }
 
-// Whole path for host-resident activations: H2D copies, then ONE launch that reads q, k, v
-// through the permutation and writes `out` in the original order (entry and exit gathers
-// fused in), then the D2H copy.  Four device buffers of one tensor each.
+// Whole path for host-resident activations.  The heads are processed in slices: the H2D copies of
+// slice c + 1 (own stream), the ONE launch of slice c (reads q, k, v through the permutation and
+// writes `out` in the original order: entry and exit gathers fused in) and the D2H copy of slice
+// c - 1 (own stream) overlap, so the two PCIe directions work at the same time.  Four device
+// buffers of one tensor each.
 extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v, void *out,
                                      hilberta_plan_t *p, void *stream) {
     if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
@@ -631,6 +640,9 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
     const int64_t dense_h = (int64_t)p->S * p->head_dim;
     if (p->stride_s != p->head_dim || p->stride_h != dense_h || p->stride_b != dense_h * p->heads)
         return HILBERTA_ERR_INVALID;
+    int dev = -1;
+    HB_CUDA(cudaGetDevice(&dev));
+    if (dev != p->device) return HILBERTA_ERR_INVALID;
     const size_t esz = p->dtype == HILBERTA_BF16 ? 2 : 4;
     const size_t bytes = (size_t)p->batch * p->heads * p->S * p->head_dim * esz;
     const size_t slot = (bytes + 255) & ~(size_t)255;
@@ -641,15 +653,45 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
         HB_CUDA(cudaMalloc(&p->ws, 4 * slot));
         p->ws_bytes = 4 * slot;
     }
+    // fp32 bindings have no slice schedule to build: chunk_heads is only set by the bf16 path
+    const int hc = (p->dtype == HILBERTA_BF16 && p->chunk_heads > 0) ? p->chunk_heads : p->heads;
+    const int n_chunks = p->heads / hc;
+    if (!p->s_in) HB_CUDA(cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking));
+    if (!p->s_out) HB_CUDA(cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking));
+    while ((int)p->ev_in.size() < n_chunks + 1) {
+        cudaEvent_t e0, e1;
+        HB_CUDA(cudaEventCreateWithFlags(&e0, cudaEventDisableTiming));
+        HB_CUDA(cudaEventCreateWithFlags(&e1, cudaEventDisableTiming));
+        p->ev_in.push_back(e0);
+        p->ev_done.push_back(e1);
+    }
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)p->ws;
     void *in[3] = {ws, ws + slot, ws + 2 * slot};
-    void *out_dev = ws + 3 * slot;
+    char *out_dev = ws + 3 * slot;
     const void *host_in[3] = {q, k, v};
-    for (int i = 0; i < 3; ++i) HB_CUDA(cudaMemcpyAsync(in[i], host_in[i], bytes, cudaMemcpyHostToDevice, st));
-    int rc = hilberta_forward_fused(in[0], in[1], in[2], out_dev, p, 1, 1, st);
-    if (rc != HILBERTA_OK) return rc;
-    HB_CUDA(cudaMemcpyAsync(out, out_dev, bytes, cudaMemcpyDeviceToHost, st));
+    // a slice of hc heads of every batch item: `batch` rows of row_bytes, one tensor of heads apart
+    const size_t row_bytes = (size_t)hc * p->S * p->head_dim * esz;
+    const size_t pitch = (size_t)p->heads * p->S * p->head_dim * esz;
+    // work already queued on the caller's stream comes first
+    HB_CUDA(cudaEventRecord(p->ev_in[n_chunks], st));
+    HB_CUDA(cudaStreamWaitEvent(p->s_in, p->ev_in[n_chunks], 0));
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t off = (size_t)c * row_bytes;
+        for (int i = 0; i < 3; ++i)
+            HB_CUDA(cudaMemcpy2DAsync((char *)in[i] + off, pitch, (const char *)host_in[i] + off, pitch, row_bytes,
+                                      p->batch, cudaMemcpyHostToDevice, p->s_in));
+        HB_CUDA(cudaEventRecord(p->ev_in[c], p->s_in));
+        HB_CUDA(cudaStreamWaitEvent(st, p->ev_in[c], 0));
+        const int rc = forward_impl(in[0], in[1], in[2], out_dev, nullptr, p, p->d_phys2orig, p->d_phys2orig, st,
+                                    n_chunks > 1 ? c : -1);
+        if (rc != HILBERTA_OK) return rc;
+        HB_CUDA(cudaEventRecord(p->ev_done[c], st));
+        HB_CUDA(cudaStreamWaitEvent(p->s_out, p->ev_done[c], 0));
+        HB_CUDA(cudaMemcpy2DAsync((char *)out + off, pitch, out_dev + off, pitch, row_bytes, p->batch,
+                                  cudaMemcpyDeviceToHost, p->s_out));
+    }
+    HB_CUDA(cudaStreamSynchronize(p->s_out));
     HB_CUDA(cudaStreamSynchronize(st));
     return HILBERTA_OK;
 }

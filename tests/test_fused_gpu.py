@@ -65,14 +65,16 @@ def test_fused_strided_inputs():
         plan.destroy()
 
 
-@pytest.mark.parametrize("D,dtype", [(128, torch.bfloat16), (64, torch.float32)])
-def test_forward_host_matches_device_path(D, dtype):
-    """Host-buffer entry point (H2D, one fused launch, D2H) against permute -> forward -> unpermute."""
+@pytest.mark.parametrize("D,dtype,B,heads", [(128, torch.bfloat16, 1, 2), (128, torch.bfloat16, 2, 6),
+                                              (128, torch.bfloat16, 1, 1), (64, torch.float32, 2, 3)])
+def test_forward_host_matches_device_path(D, dtype, B, heads):
+    """Host-buffer entry point (copies and fused launches pipelined over slices of heads) against
+    permute -> forward -> unpermute."""
     H = W = 32
-    nt, heads = 21, 2
+    nt = 21
     S = nt + H * W
     g = torch.Generator().manual_seed(79)
-    q, k, v = (torch.randn((1, heads, S, D), generator=g).to(dtype).pin_memory() for _ in range(3))
+    q, k, v = (torch.randn((B, heads, S, D), generator=g).to(dtype).pin_memory() for _ in range(3))
     out_h = torch.empty_like(q).pin_memory()
     plan = hb.Plan(H, W, 256, 192, 4, nt)
     try:
