@@ -65,12 +65,16 @@ def _run(H, W, tile, o, hs, nt, B, heads, groups=0, q_gain=1.0, seed=5):
     (16, 16, 256, 0, 0, 0, 1, 2, 0),        # one tile, no shared region: dense attention
     (32, 32, 0, 37, 4, 50, 1, 2, 6),        # equal groups over the non-shared tokens (Appendix A)
     (16, 16, 64, 0, 16, 3, 1, 1, 0),        # every image token shared: prefix rows only
+    (1, 1, 1, 0, 0, 0, 1, 1, 0),            # a single token
+    (2, 2, 4, 1, 0, 300, 1, 2, 0),          # four image tokens behind 300 text tokens
+    (8, 8, 2, 1, 2, 0, 1, 1, 0),            # 32 tiles of two positions each
 ])
 def test_backward_matches_oracle(H, W, tile, o, hs, nt, B, heads, groups):
     got, ref = _run(H, W, tile, o, hs, nt, B, heads, groups)
     for name, g, r in zip(("dq", "dk", "dv"), got, ref):
         assert np.isfinite(g).all(), name
-        assert orc.rel_l2_err(g, r) <= 5e-3, (name, orc.rel_l2_err(g, r))
+        if np.abs(r).max() > 0:   # a lone token has dq = dk = 0 exactly; only the absolute bar applies
+            assert orc.rel_l2_err(g, r) <= 5e-3, (name, orc.rel_l2_err(g, r))
         assert orc.max_abs_err(g, r) <= 1e-2 * max(1.0, np.abs(r).max()), (name, orc.max_abs_err(g, r))
 
 
