@@ -199,6 +199,7 @@ def main():
                     help="use the Appendix-A tiling with this many equal groups over the non-shared tokens "
                          "(the paper's Table 1 settings: --groups 4|16 --shared 16 at 1024^2, 32 at 2048^2)")
     ap.add_argument("--shared", type=int, default=-1, help="override the side of the central shared region")
+    ap.add_argument("--head-dim", type=int, default=0, help="override the head dim (bf16: 128 or 64)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the dense / SDPA context rows")
@@ -215,6 +216,8 @@ def main():
         wl = wl.with_(tile=args.tile, layer_offset=args.tile // 2)
     if args.shared >= 0:
         wl = wl.with_(shared_region=args.shared)
+    if args.head_dim:
+        wl = wl.with_(head_dim=args.head_dim)
     if args.groups:
         if args.impl == "reference" or args.schedule:
             raise SystemExit("--groups is a timing-only option of the CUDA arm")
@@ -406,7 +409,7 @@ def main():
 
     # ---- backward pass (not part of the metric): dq, dk, dv on the same plan and inputs
     backward = None
-    if world == 1 and not args.no_backward and wl.dtype == "bf16":
+    if world == 1 and not args.no_backward and wl.dtype == "bf16" and wl.head_dim == 128:
         lse = torch.empty((wl.batch, wl.heads, wl.S), device="cuda", dtype=torch.float32)
         g = torch.Generator().manual_seed(wl.seed + 7)
         dop = torch.randn(qp.shape, generator=g).to(torch.bfloat16).cuda()

@@ -140,7 +140,7 @@ int hilberta_plan_export(const hilberta_plan_t *plan, int what, void *host_buf, 
  * configuration line: batch Z, heads, head dim D, softmax scale s, strides).
  *
  *   batch, heads   >= 1.  The same mask serves every (batch, head).
- *   head_dim       bf16: 128.  fp32: 32, 64 or 128.  Others: ERR_UNSUPPORTED.
+ *   head_dim       bf16: 128 or 64.  fp32: 32, 64 or 128.  Others: ERR_UNSUPPORTED.
  *   dtype          HILBERTA_BF16 (tensor-core kernel) or HILBERTA_FP32 (plain FMA kernel).
  *   stride_b, stride_h, stride_s
  *                  element strides of q, k, v and out (all four share them) for
@@ -199,8 +199,8 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  * the same plan must not overlap on the device.
  *
  * Errors: ERR_INVALID (NULL, misaligned or aliasing pointers, wrong device),
- * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding: only the bf16 tensor-core path has a
- * backward pass), ERR_CUDA. */
+ * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding, or head_dim 64: only the bf16
+ * tensor-core path with head_dim 128 has a backward pass), ERR_CUDA. */
 int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                       const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
                       void *stream);

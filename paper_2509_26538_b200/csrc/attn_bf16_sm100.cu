@@ -41,14 +41,14 @@ namespace {
 
 constexpr int BM = 128;        // rows per query tile
 constexpr int BN = 128;        // keys per block
-constexpr int HD = 128;        // head dim
 constexpr int QT = 2;          // query tiles per work item
 constexpr int ITEM_ROWS = QT * BM;
 constexpr int NSTAGE = 5;      // K/V ring slots (K0 V0 K1 V1 ...)
-constexpr int TILE_BYTES = BN * HD * 2;  // 32 KB: two 64-column slabs of 128 rows
-constexpr int SLAB_BYTES = TILE_BYTES / 2;
+constexpr int SLAB_BYTES = BN * 128;     // one 64-column slab of 128 rows (128-byte swizzled rows)
+// head dim HD = 128: a tile is two slabs (32 KB); HD = 64: one slab (16 KB)
+__host__ __device__ constexpr int tile_bytes(int hd) { return BN * hd * 2; }
 constexpr int THREADS = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle (register donors)
-constexpr int SMEM_BYTES = (QT + NSTAGE) * TILE_BYTES + 1024;
+__host__ __device__ constexpr int smem_bytes(int hd) { return (QT + NSTAGE) * tile_bytes(hd) + 1024; }
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 #ifndef HB_POLY_MASK
@@ -126,6 +126,7 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
 }
 
 // S_t = Q_t K^T for one 128-key block: 8 MMAs of K = 16.
+template <int HD>
 __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t sQt, uint32_t sKslot) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, BN, 0, 0);
     // the start-address field is the low 14 bits (16-byte units): stepping K is one add
@@ -139,6 +140,7 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t sQt, uint32_t
 
 // O_t (+)= P_t V for one 128-key block: P from TMEM, V row-major in smem (N-major operand).
 // `half` selects keys [64 half, +64) of the block: four MMAs of K = 16.
+template <int HD>
 __device__ __forceinline__ void issue_pv_half(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, int half,
                                               bool accumulate) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
@@ -160,7 +162,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int sr
 // GATHER = true : the tensors are in ORIGINAL order (the entry gather of Sec. 3.4 fused in): two loader
 // warps fetch every tile row through the permutation table with 16-byte cp.async copies and place it
 // where a 128-byte-swizzled TMA box would have put it, so everything downstream is unchanged.
-template <bool GATHER>
+template <bool GATHER, int HD>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const KernelParams<GATHER> prm) {
@@ -168,6 +170,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __shared__ uint64_t bars[NUM_BARS];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    constexpr int TILE_BYTES = tile_bytes(HD);
+    constexpr int NSLAB = HD / 64;
 
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sQ = smem_u32(smem);
@@ -206,8 +210,6 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if constexpr (GATHER) {
     if (warp == 10 || warp == 11) {
         // ------------------------------------------------- gathering loaders (entry permute fused in)
-        const int lt = tid - 10 * 32;        // 0 .. 63
-        const int chunk = lt & 15;           // 16-byte piece of a 256-byte row
         uint32_t kvc = 0, qc = 0;
         bool ok = true;
         // The stage's barrier counts one arrival per loader thread; each arrival fires by itself
@@ -215,13 +217,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         auto publish = [&](uint32_t b) {
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(b) : "memory");
         };
-        // Warp w of the two copies rows [64 w, 64 w + 64) of a tile, two adjacent rows per
-        // instruction (lanes 0-15 one row, lanes 16-31 the next; 16 bytes per lane).  Lane L fetches
-        // the table entries of rows L and 32 + L of that range once per tile; the lanes that copy a
+        // Warp w of the two copies rows [64 w, 64 w + 64) of a tile, RPI adjacent rows per
+        // instruction (16 bytes per lane; a row is CH = HD / 8 lanes wide).  Lane L fetches the
+        // table entries of rows L and 32 + L of that range once per tile; the lanes that copy a
         // row pick its entry up by shuffle, so the table costs one load latency per tile.
-        const int lane = tid & 31, half = lane >> 4, wrow = (warp - 10) * 64;
-        const uint32_t dst_lane = (uint32_t)((chunk >> 3) * SLAB_BYTES + (wrow + half) * 128);
-        const int c7 = (chunk & 7) ^ half;   // row & 7 = (2 i + half) & 7 = (2 i & 7) ^ half
+        constexpr int CH = HD / 8, RPI = 32 / CH;
+        const int lane = tid & 31, chunk = lane % CH, sub = lane / CH, wrow = (warp - 10) * 64;
+        const uint32_t dst_lane = (uint32_t)((chunk >> 3) * SLAB_BYTES + (wrow + sub) * 128);
+        const int c7 = (chunk & 7) ^ sub;   // row & 7 = (RPI i + sub) & 7 = ((RPI i) & 7) ^ sub
         auto load_rows = [&](int row0, int &ia, int &ib) {
             const int pa = row0 + wrow + lane, pb = pa + 32;
             ia = pa < prm.S ? __ldg(prm.in_map + pa) : -1;   // rows beyond the sequence are
@@ -231,9 +234,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const __nv_bfloat16 *src0 = base + chunk * 8;
             const uint32_t dst0 = dst_tile + dst_lane;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int orow = __shfl_sync(0xffffffffu, i < 16 ? ia : ib, ((2 * i) & 31) + half);
-                const uint32_t dst = dst0 + i * 256 + ((c7 ^ ((2 * i) & 7)) << 4);
+            for (int i = 0; i < 64 / RPI; ++i) {
+                const int orow = __shfl_sync(0xffffffffu, RPI * i < 32 ? ia : ib, ((RPI * i) & 31) + sub);
+                const uint32_t dst = dst0 + i * (RPI * 128) + ((c7 ^ ((RPI * i) & 7)) << 4);
                 cp_async16(dst, src0 + (long long)max(orow, 0) * prm.stride_s, orow >= 0 ? 16 : 0);
             }
         };
@@ -272,7 +275,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         copy_tile(sKV + s * TILE_BYTES, (kv ? prm.gv : prm.gk) + bh_off, ia, ib);
                         publish(bar(KV_FULL + s));
 #ifdef HB_TIMING
-                        if (lt == 0) {
+                        if (tid == 10 * 32) {
                             atomicAdd(prm.status + 24, (int)((tg1 - tg0) >> 4));
                             atomicAdd(prm.status + 25, (int)((clock64() - tg1) >> 4));
                             atomicAdd(prm.status + 26, 1);
@@ -305,8 +308,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 ++qc;
                 mbar_expect_tx(bar(Q_FULL), nt * TILE_BYTES);
                 for (int t = 0; t < nt; ++t) {
-                    tma_load_4d(sQ + t * TILE_BYTES, &tmQ, bar(Q_FULL), 0, wi.q_start + t * BM, h, b);
-                    tma_load_4d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, bar(Q_FULL), 64, wi.q_start + t * BM, h, b);
+#pragma unroll
+                    for (int sl = 0; sl < NSLAB; ++sl)
+                        tma_load_4d(sQ + t * TILE_BYTES + sl * SLAB_BYTES, &tmQ, bar(Q_FULL), 64 * sl,
+                                    wi.q_start + t * BM, h, b);
                 }
                 for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                     const int nb = item_blocks(wi, seg);
@@ -319,8 +324,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                             if (!ok) break;
                             const CUtensorMap *tm = kv ? &tmV : &tmK;
                             mbar_expect_tx(bar(KV_FULL + s), TILE_BYTES);
-                            tma_load_4d(sKV + s * TILE_BYTES, tm, bar(KV_FULL + s), 0, row, h, b);
-                            tma_load_4d(sKV + s * TILE_BYTES + SLAB_BYTES, tm, bar(KV_FULL + s), 64, row, h, b);
+#pragma unroll
+                            for (int sl = 0; sl < NSLAB; ++sl)
+                                tma_load_4d(sKV + s * TILE_BYTES + sl * SLAB_BYTES, tm, bar(KV_FULL + s), 64 * sl, row, h, b);
                         }
                         if (!ok) break;
                     }
@@ -360,7 +366,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t) {
-                    issue_qk(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
+                    issue_qk<HD>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
                     mma_commit(bar(S_FULL + t));
                 }
                 mma_commit(bar(KV_EMPTY + slot_of(2 * g)));
@@ -392,7 +398,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef HB_TIMING
                         tm_p += clock64() - tp0;
 #endif
-                        issue_pv_half(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
+                        issue_pv_half<HD>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
 #ifdef HB_TIMING
                         const long long tp1 = clock64();
 #endif
@@ -403,10 +409,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         tm_p += clock64() - tp1;
 #endif
                         tc_fence_after();
-                        issue_pv_half(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
+                        issue_pv_half<HD>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
                         mma_commit(bar(PV_DONE + t));
                         if (more) {
-                            issue_qk(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
+                            issue_qk<HD>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
                             mma_commit(bar(S_FULL + t));
                         }
                     }
@@ -656,7 +662,7 @@ int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, 
     if (heads <= 0) heads = p->heads;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return HILBERTA_ERR_CUDA;
-    cuuint64_t dims[4] = {128, (cuuint64_t)p->S, (cuuint64_t)heads, (cuuint64_t)p->batch};
+    cuuint64_t dims[4] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->S, (cuuint64_t)heads, (cuuint64_t)p->batch};
     cuuint64_t strides[3] = {(cuuint64_t)p->stride_s * 2, (cuuint64_t)p->stride_h * 2, (cuuint64_t)p->stride_b * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -788,10 +794,16 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128));
         if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            SMEM_BYTES);
+            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            smem_bytes(128));
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            smem_bytes(64));
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            smem_bytes(64));
     });
     HB_CUDA(attr_err);
     return HILBERTA_OK;
@@ -843,11 +855,17 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
         gprm.gq = (const __nv_bfloat16 *)q;
         gprm.gk = (const __nv_bfloat16 *)k;
         gprm.gv = (const __nv_bfloat16 *)v;
-        attn_bf16_kernel<true><<<n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, gprm);
+        if (p->head_dim == 128)
+            attn_bf16_kernel<true, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, gprm);
+        else
+            attn_bf16_kernel<true, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, gprm);
     } else {
         KernelParams<false> pprm;
         static_cast<Params &>(pprm) = prm;
-        attn_bf16_kernel<false><<<n_cta, THREADS, SMEM_BYTES, stream>>>(mq, mk, mv, pprm);
+        if (p->head_dim == 128)
+            attn_bf16_kernel<false, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, pprm);
+        else
+            attn_bf16_kernel<false, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, pprm);
     }
     HB_LAUNCHED();
     return HILBERTA_OK;

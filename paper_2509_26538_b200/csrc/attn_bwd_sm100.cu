@@ -714,7 +714,7 @@ extern "C" int hilberta_backward_static(const void *dout, const void *q, const v
                                         const hilberta_plan_t *p, void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
+    if (p->dtype != HILBERTA_BF16 || p->head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = ((uintptr_t)lse & 3) ? 15 : 0;

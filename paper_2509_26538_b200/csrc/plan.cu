@@ -536,7 +536,7 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
                                   int64_t stride_b, int64_t stride_h, int64_t stride_s, float scale) {
     if (!p || batch < 1 || heads < 1 || head_dim < 1) return HILBERTA_ERR_INVALID;
     if (dtype != HILBERTA_BF16 && dtype != HILBERTA_FP32) return HILBERTA_ERR_INVALID;
-    if (dtype == HILBERTA_BF16 && head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
+    if (dtype == HILBERTA_BF16 && head_dim != 128 && head_dim != 64) return HILBERTA_ERR_UNSUPPORTED;
     if (dtype == HILBERTA_FP32 && head_dim != 32 && head_dim != 64 && head_dim != 128)
         return HILBERTA_ERR_UNSUPPORTED;
     if (stride_b == 0 && stride_h == 0 && stride_s == 0) {
@@ -559,8 +559,10 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
     if (dtype == HILBERTA_BF16) {
         int rc = attn_bf16_prepare(p);
         if (rc != HILBERTA_OK) return rc;
-        rc = attn_bwd_prepare(p);
-        if (rc != HILBERTA_OK) return rc;
+        if (head_dim == 128) {   // the backward pass exists for head dim 128 only
+            rc = attn_bwd_prepare(p);
+            if (rc != HILBERTA_OK) return rc;
+        }
     }
     p->bound = true;
     return HILBERTA_OK;
@@ -609,7 +611,7 @@ extern "C" int hilberta_backward(const void *dout, const void *q, const void *k,
                                  void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
+    if (p->dtype != HILBERTA_BF16 || p->head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = (uintptr_t)lse & 3 ? 15 : 0;
