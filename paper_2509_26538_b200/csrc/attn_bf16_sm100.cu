@@ -706,7 +706,7 @@ int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
 }
 
 // Static schedule: every (item, batch*head) unit goes to the least-loaded CTA, longest units
-// first (cost = MMA block pairs + a fixed per-unit overhead); units are stored grouped by CTA.
+// first (cost = tile-blocks + a fixed per-unit overhead); units are stored grouped by CTA.
 static int upload_schedule(const std::vector<WorkItem> &items, int bh, int sm_count, WorkUnit **d_units,
                            int **d_cta_begin, int *n_cta_out) {
     const long long n_units = (long long)items.size() * bh;
@@ -717,7 +717,9 @@ static int upload_schedule(const std::vector<WorkItem> &items, int bh, int sm_co
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
     for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
     for (int i = 0; i < (int)items.size(); ++i) {
-        const long long cost = (long long)items[i].kv_blocks * (items[i].q_rows > BM ? 2 : 1) + 2;
+        // a unit with one query tile has no second tile to overlap its softmax with the MMAs: its
+        // blocks take about 1.3 x half the time of a two-tile unit's (in tenths of a tile-block)
+        const long long cost = (long long)items[i].kv_blocks * (items[i].q_rows > BM ? 20 : 13) + 20;
         for (int j = 0; j < bh; ++j) {
             Load top = heap.top();
             heap.pop();
@@ -756,8 +758,8 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
         if (w.seg1_len > 0) add_items(items, w.seg1_start, w.seg1_len, 3, st, ln);
     }
     std::stable_sort(items.begin(), items.end(), [](const WorkItem &a, const WorkItem &b) {
-        const long long ca = (long long)a.kv_blocks * (a.q_rows > BM ? 2 : 1);
-        const long long cb = (long long)b.kv_blocks * (b.q_rows > BM ? 2 : 1);
+        const long long ca = (long long)a.kv_blocks * (a.q_rows > BM ? 20 : 13);
+        const long long cb = (long long)b.kv_blocks * (b.q_rows > BM ? 20 : 13);
         return ca > cb;
     });
     cudaFree(p->d_work);
