@@ -513,29 +513,45 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
     }
 }
 
-// lse2[row] = lse[row] * log2 e, delta[row] = sum_d dO[row, d] * O[row, d]: one warp per row, 8 bytes per lane.
+// lse2[row] = lse[row] * log2 e, delta[row] = sum_d dO[row, d] * O[row, d]: sixteen lanes per row
+// (16 bytes each of the 256-byte row), two rows per warp, four rows in flight per thread group.
 __global__ void __launch_bounds__(256)
 delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__restrict__ out,
              const float *__restrict__ lse, float *__restrict__ lse2, float *__restrict__ delta, int S, int heads,
              long long stride_b, long long stride_h, long long stride_s, long long n_rows) {
-    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (row >= n_rows) return;
-    const int lane = threadIdx.x & 31;
-    const long long bh = row / S;
-    const int r = (int)(row % S);
-    const long long off = (bh / heads) * stride_b + (bh % heads) * stride_h + (long long)r * stride_s + lane * 4;
-    const uint2 a = *reinterpret_cast<const uint2 *>(dout + off);
-    const uint2 c = *reinterpret_cast<const uint2 *>(out + off);
-    const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&a.x));
-    const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&a.y));
-    const float2 c0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&c.x));
-    const float2 c1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&c.y));
-    float acc = a0.x * c0.x + a0.y * c0.y + a1.x * c1.x + a1.y * c1.y;
+    const int sub = threadIdx.x & 15;
+    const long long row0 = ((long long)blockIdx.x * 16 + (threadIdx.x >> 4)) * 4;
+    uint4 a[4], c[4];
+    bool in[4];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) {
-        lse2[row] = lse[row] * 1.4426950408889634f;
-        delta[row] = acc;
+    for (int i = 0; i < 4; ++i) {
+        const long long row = row0 + i;
+        in[i] = row < n_rows;
+        if (in[i]) {
+            const long long bh = row / S;
+            const long long off = (bh / heads) * stride_b + (bh % heads) * stride_h + (row % S) * stride_s + sub * 8;
+            a[i] = *reinterpret_cast<const uint4 *>(dout + off);
+            c[i] = *reinterpret_cast<const uint4 *>(out + off);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float acc = 0.f;
+        if (in[i]) {
+            const uint32_t *ua = reinterpret_cast<const uint32_t *>(&a[i]), *uc = reinterpret_cast<const uint32_t *>(&c[i]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ua[e]));
+                const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&uc[e]));
+                acc = fmaf(x.x, y.x, fmaf(x.y, y.y, acc));
+            }
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (in[i] && sub == 0) {
+            lse2[row0 + i] = lse[row0 + i] * 1.4426950408889634f;
+            delta[row0 + i] = acc;
+        }
     }
 }
 
@@ -645,7 +661,7 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
     if ((rc = make_tensor_map(&mv, v, p, BK)) != HILBERTA_OK) return rc;
     if ((rc = make_tensor_map(&mdo, dout, p, BK)) != HILBERTA_OK) return rc;
     const long long n_rows = (long long)p->batch * p->heads * p->S;
-    delta_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, stream>>>(
+    delta_kernel<<<(unsigned)((n_rows + 63) / 64), 256, 0, stream>>>(
         (const __nv_bfloat16 *)dout, (const __nv_bfloat16 *)out, lse, delta, delta + n_rows, p->S, p->heads,
         p->stride_b, p->stride_h, p->stride_s, n_rows);
     HB_LAUNCHED();
