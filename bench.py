@@ -409,7 +409,7 @@ def main():
 
     # ---- backward pass (not part of the metric): dq, dk, dv on the same plan and inputs
     backward = None
-    if world == 1 and not args.no_backward and wl.dtype == "bf16" and wl.head_dim == 128:
+    if world == 1 and not args.no_backward and wl.dtype == "bf16":
         lse = torch.empty((wl.batch, wl.heads, wl.S), device="cuda", dtype=torch.float32)
         g = torch.Generator().manual_seed(wl.seed + 7)
         dop = torch.randn(qp.shape, generator=g).to(torch.bfloat16).cuda()

@@ -199,8 +199,8 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  * the same plan must not overlap on the device.
  *
  * Errors: ERR_INVALID (NULL, misaligned or aliasing pointers, wrong device),
- * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding, or head_dim 64: only the bf16
- * tensor-core path with head_dim 128 has a backward pass), ERR_CUDA. */
+ * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding: only the bf16 tensor-core path has a
+ * backward pass), ERR_CUDA. */
 int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                       const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
                       void *stream);

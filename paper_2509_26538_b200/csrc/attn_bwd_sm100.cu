@@ -42,8 +42,7 @@ namespace {
 
 constexpr int BM = 128;   // resident rows per work item
 constexpr int BK = 128;   // streamed rows per block
-constexpr int HD = 128;
-constexpr int TILE_BYTES = BM * HD * 2;   // 32 KB: two 64-column slabs of 128 rows
+constexpr int TILE_BYTES = BM * 128 * 2;  // 32 KB slot: two 64-column slabs of 128 rows (head dim 64 uses the first)
 constexpr int SLAB_BYTES = TILE_BYTES / 2;
 constexpr int NT1 = 3;    // ring of the streamed operand that is read twice (scores early, output MMA late)
 constexpr int NT2 = 2;    // ring of the streamed operand of dP
@@ -96,6 +95,7 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
 }
 
 // acc = R T^T: resident tile (128 rows) times a streamed block (128 rows), K = head dim.
+template <int HD>
 __device__ __forceinline__ void issue_rt(uint32_t tmem_acc, uint32_t sR, uint32_t sT) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, BK, 0, 0);
     const uint64_t da = smem_desc_sw128(sR, 16, 1024), db = smem_desc_sw128(sT, 16, 1024);
@@ -109,6 +109,7 @@ __device__ __forceinline__ void issue_rt(uint32_t tmem_acc, uint32_t sR, uint32_
 // out (+)= A T: A (128 x 128, bf16) from TMEM, the streamed block row-major in smem (N-major
 // operand: 128 rows of K, two 64-column slabs of N).  The bf16 pairs of streamed rows
 // [32 g, 32 g + 32) sit 16 columns wide at column 32 g of region B (+ a_off).
+template <int HD>
 __device__ __forceinline__ void issue_at(uint32_t tmem_out, uint32_t tmem_b, uint32_t a_off, uint32_t sT,
                                          bool accumulate) {
     constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
@@ -119,13 +120,15 @@ __device__ __forceinline__ void issue_at(uint32_t tmem_out, uint32_t tmem_b, uin
                (accumulate || k > 0) ? 1u : 0u);
 }
 
-template <int MODE>
+template <int MODE, int HD>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant__ CUtensorMap tmR2,
                 const __grid_constant__ CUtensorMap tmT1, const __grid_constant__ CUtensorMap tmT2,
                 const Params prm) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t REG_A = 0, REG_B = 128, OUT_A = 256, OUT_B = 384;   // TMEM columns
+    constexpr int NSLAB = HD / 64;
+    constexpr uint32_t TILE_TX = BM * HD * 2;                              // bytes of one tile
 
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     if ((int)(smem - smem_raw) + SMEM_USED > SMEM_BYTES) {
@@ -197,9 +200,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                         if (!ok) break;
                         if (leader) {
                             const uint32_t dst = ring + s * TILE_BYTES;
-                            mbar_expect_tx(bar(FULL + s), TILE_BYTES);
-                            tma_load_4d(dst, tm, bar(FULL + s), 0, row, h, b);
-                            tma_load_4d(dst + SLAB_BYTES, tm, bar(FULL + s), 64, row, h, b);
+                            mbar_expect_tx(bar(FULL + s), TILE_TX);
+#pragma unroll
+                            for (int sl = 0; sl < NSLAB; ++sl)
+                                tma_load_4d(dst + sl * SLAB_BYTES, tm, bar(FULL + s), 64 * sl, row, h, b);
                         }
                         if (with_stats) {
                             // lse2 and delta of the block's rows that lie inside the range (the others
@@ -244,20 +248,22 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                 // free once the last R T^T MMA of the previous unit has retired
                 if (uc > 0) ok = wait_or_abort(bar(RES_EMPTY), (uc - 1) & 1, abort_flag, prm.status, 0x401);
                 if (!ok) break;
-                mbar_expect_tx(bar(RES_FULL), 2 * TILE_BYTES);
-                tma_load_4d(sR1, &tmR1, bar(RES_FULL), 0, wi.q_start, h, b);
-                tma_load_4d(sR1 + SLAB_BYTES, &tmR1, bar(RES_FULL), 64, wi.q_start, h, b);
-                tma_load_4d(sR2, &tmR2, bar(RES_FULL), 0, wi.q_start, h, b);
-                tma_load_4d(sR2 + SLAB_BYTES, &tmR2, bar(RES_FULL), 64, wi.q_start, h, b);
+                mbar_expect_tx(bar(RES_FULL), 2 * TILE_TX);
+#pragma unroll
+                for (int sl = 0; sl < NSLAB; ++sl) {
+                    tma_load_4d(sR1 + sl * SLAB_BYTES, &tmR1, bar(RES_FULL), 64 * sl, wi.q_start, h, b);
+                    tma_load_4d(sR2 + sl * SLAB_BYTES, &tmR2, bar(RES_FULL), 64 * sl, wi.q_start, h, b);
+                }
                 if (u + 1 < u_end) {
                     // pull the next unit's resident tiles into L2 while this unit runs
                     const WorkUnit nu = prm.units[u + 1];
                     const int nq = prm.work[nu.item].q_start;
                     const int nb_ = nu.bh / prm.heads, nh = nu.bh % prm.heads;
-                    tma_prefetch_4d(&tmR1, 0, nq, nh, nb_);
-                    tma_prefetch_4d(&tmR1, 64, nq, nh, nb_);
-                    tma_prefetch_4d(&tmR2, 0, nq, nh, nb_);
-                    tma_prefetch_4d(&tmR2, 64, nq, nh, nb_);
+#pragma unroll
+                    for (int sl = 0; sl < NSLAB; ++sl) {
+                        tma_prefetch_4d(&tmR1, 64 * sl, nq, nh, nb_);
+                        tma_prefetch_4d(&tmR2, 64 * sl, nq, nh, nb_);
+                    }
                 }
             }
             if (!ok) {
@@ -283,15 +289,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
             tc_fence_after();
             const long long roff = (long long)b * prm.stride_b + (long long)h * prm.stride_h +
                                    (long long)(wi.q_start + r) * prm.stride_s;
-            constexpr int NCH = (MODE == MODE_DKV) ? 8 : 4;   // DKV: dK then dV
+            constexpr int CPO = HD / 32;                              // 32-column chunks per output
+            constexpr int NCH = (MODE == MODE_DKV) ? 2 * CPO : CPO;   // DKV: dK then dV
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 uint32_t o[32];
-                tmem_ld32(tmem + lane_addr + OUT_A + c * 32, o);
+                tmem_ld32(tmem + lane_addr + (c >= CPO ? OUT_B + (c - CPO) * 32 : OUT_A + c * 32), o);
                 tmem_wait_ld();
                 if (row_ok) {
-                    __nv_bfloat16 *orow = (c >= 4 ? prm.out_b : prm.out_a) + roff + (c & 3) * 32;
-                    const float mul = c >= 4 ? 1.f : prm.scale;
+                    __nv_bfloat16 *orow = (c >= CPO ? prm.out_b : prm.out_a) + roff + (c % CPO) * 32;
+                    const float mul = c >= CPO ? 1.f : prm.scale;
                     uint32_t w[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
@@ -325,12 +332,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                 ok = wait_or_abort(bar(T1_FULL + g % NT1), (g / NT1) & 1, abort_flag, prm.status, 0x502);
                 if (!ok) break;
                 tc_fence_after();
-                issue_rt(tmem + REG_A, sR1, t1(g));
+                issue_rt<HD>(tmem + REG_A, sR1, t1(g));
                 mma_commit(bar(S_FULL));
                 ok = wait_or_abort(bar(T2_FULL + g % NT2), (g / NT2) & 1, abort_flag, prm.status, 0x503);
                 if (!ok) break;
                 tc_fence_after();
-                issue_rt(tmem + REG_B, sR2, t2(g));
+                issue_rt<HD>(tmem + REG_B, sR2, t2(g));
                 mma_commit(bar(DP_FULL));
                 if (MODE == MODE_DQ) mma_commit(bar(T2_EMPTY + g % NT2));
                 if (n == 1) mma_commit(bar(RES_EMPTY));
@@ -344,7 +351,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                         ok = wait_or_abort(bar(A_DONE), e & 1, abort_flag, prm.status, 0x505);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_rt(tmem + REG_A, sR1, t1(e + 1));
+                        issue_rt<HD>(tmem + REG_A, sR1, t1(e + 1));
                         mma_commit(bar(S_FULL));
                     }
                     if (s == 0 && uc > 0) {
@@ -355,8 +362,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                     ok = wait_or_abort(bar(P_READY), e & 1, abort_flag, prm.status, 0x507);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_at(tmem + OUT_A, tmem + REG_B, 16, t1(e), s > 0);                       // dS  x T1
-                    if (MODE == MODE_DKV) issue_at(tmem + OUT_B, tmem + REG_B, 0, t2(e), s > 0);   // P^T x T2
+                    issue_at<HD>(tmem + OUT_A, tmem + REG_B, 16, t1(e), s > 0);                       // dS  x T1
+                    if (MODE == MODE_DKV) issue_at<HD>(tmem + OUT_B, tmem + REG_B, 0, t2(e), s > 0);   // P^T x T2
                     mma_commit(bar(T1_EMPTY + e % NT1));
                     if (MODE == MODE_DKV) mma_commit(bar(T2_EMPTY + e % NT2));
                     if (more) {
@@ -364,7 +371,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                         ok = wait_or_abort(bar(T2_FULL + (e + 1) % NT2), ((e + 1) / NT2) & 1, abort_flag, prm.status, 0x508);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_rt(tmem + REG_B, sR2, t2(e + 1));
+                        issue_rt<HD>(tmem + REG_B, sR2, t2(e + 1));
                         mma_commit(bar(DP_FULL));
                         if (MODE == MODE_DQ) mma_commit(bar(T2_EMPTY + (e + 1) % NT2));
                         if (s + 2 == n) mma_commit(bar(RES_EMPTY));   // last read of the resident tiles
@@ -513,14 +520,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
     }
 }
 
-// lse2[row] = lse[row] * log2 e, delta[row] = sum_d dO[row, d] * O[row, d]: sixteen lanes per row
-// (16 bytes each of the 256-byte row), two rows per warp, four rows in flight per thread group.
+// lse2[row] = lse[row] * log2 e, delta[row] = sum_d dO[row, d] * O[row, d]: HD / 8 lanes per row
+// (16 bytes each), four rows in flight per lane group.
+template <int HD>
 __global__ void __launch_bounds__(256)
 delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__restrict__ out,
              const float *__restrict__ lse, float *__restrict__ lse2, float *__restrict__ delta, int S, int heads,
              long long stride_b, long long stride_h, long long stride_s, long long n_rows) {
-    const int sub = threadIdx.x & 15;
-    const long long row0 = ((long long)blockIdx.x * 16 + (threadIdx.x >> 4)) * 4;
+    constexpr int LPR = HD / 8;   // lanes per row (16 bytes each)
+    const int sub = threadIdx.x % LPR;
+    const long long row0 = ((long long)blockIdx.x * (256 / LPR) + threadIdx.x / LPR) * 4;
     uint4 a[4], c[4];
     bool in[4];
 #pragma unroll
@@ -547,7 +556,7 @@ delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__rest
             }
         }
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (in[i] && sub == 0) {
             lse2[row0 + i] = lse[row0 + i] * 1.4426950408889634f;
             delta[row0 + i] = acc;
@@ -641,10 +650,10 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bwd_kernel<MODE_DKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            SMEM_BYTES);
+        const void *kernels[4] = {(const void *)attn_bwd_kernel<MODE_DQ, 128>, (const void *)attn_bwd_kernel<MODE_DKV, 128>,
+                                  (const void *)attn_bwd_kernel<MODE_DQ, 64>, (const void *)attn_bwd_kernel<MODE_DKV, 64>};
+        for (int i = 0; i < 4 && attr_err == cudaSuccess; ++i)
+            attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     });
     HB_CUDA(attr_err);
     return HILBERTA_OK;
@@ -661,9 +670,14 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
     if ((rc = make_tensor_map(&mv, v, p, BK)) != HILBERTA_OK) return rc;
     if ((rc = make_tensor_map(&mdo, dout, p, BK)) != HILBERTA_OK) return rc;
     const long long n_rows = (long long)p->batch * p->heads * p->S;
-    delta_kernel<<<(unsigned)((n_rows + 63) / 64), 256, 0, stream>>>(
-        (const __nv_bfloat16 *)dout, (const __nv_bfloat16 *)out, lse, delta, delta + n_rows, p->S, p->heads,
-        p->stride_b, p->stride_h, p->stride_s, n_rows);
+    if (p->head_dim == 128)
+        delta_kernel<128><<<(unsigned)((n_rows + 63) / 64), 256, 0, stream>>>(
+            (const __nv_bfloat16 *)dout, (const __nv_bfloat16 *)out, lse, delta, delta + n_rows, p->S, p->heads,
+            p->stride_b, p->stride_h, p->stride_s, n_rows);
+    else
+        delta_kernel<64><<<(unsigned)((n_rows + 127) / 128), 256, 0, stream>>>(
+            (const __nv_bfloat16 *)dout, (const __nv_bfloat16 *)out, lse, delta, delta + n_rows, p->S, p->heads,
+            p->stride_b, p->stride_h, p->stride_s, n_rows);
     HB_LAUNCHED();
     Params prm;
     prm.work = p->d_bwd_work;
@@ -683,11 +697,17 @@ int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, c
                        ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
     prm.out_a = (__nv_bfloat16 *)dq;
     prm.out_b = nullptr;
-    attn_bwd_kernel<MODE_DQ><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mq, mdo, mk, mv, prm);
+    if (p->head_dim == 128)
+        attn_bwd_kernel<MODE_DQ, 128><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mq, mdo, mk, mv, prm);
+    else
+        attn_bwd_kernel<MODE_DQ, 64><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mq, mdo, mk, mv, prm);
     HB_LAUNCHED();
     prm.out_a = (__nv_bfloat16 *)dk;
     prm.out_b = (__nv_bfloat16 *)dv;
-    attn_bwd_kernel<MODE_DKV><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mk, mv, mq, mdo, prm);
+    if (p->head_dim == 128)
+        attn_bwd_kernel<MODE_DKV, 128><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mk, mv, mq, mdo, prm);
+    else
+        attn_bwd_kernel<MODE_DKV, 64><<<p->n_bwd_cta, THREADS, SMEM_BYTES, stream>>>(mk, mv, mq, mdo, prm);
     HB_LAUNCHED();
     return HILBERTA_OK;
 }
@@ -730,7 +750,7 @@ extern "C" int hilberta_backward_static(const void *dout, const void *q, const v
                                         const hilberta_plan_t *p, void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (p->dtype != HILBERTA_BF16 || p->head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
+    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = ((uintptr_t)lse & 3) ? 15 : 0;

@@ -559,10 +559,8 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
     if (dtype == HILBERTA_BF16) {
         int rc = attn_bf16_prepare(p);
         if (rc != HILBERTA_OK) return rc;
-        if (head_dim == 128) {   // the backward pass exists for head dim 128 only
-            rc = attn_bwd_prepare(p);
-            if (rc != HILBERTA_OK) return rc;
-        }
+        rc = attn_bwd_prepare(p);
+        if (rc != HILBERTA_OK) return rc;
     }
     p->bound = true;
     return HILBERTA_OK;
@@ -611,7 +609,7 @@ extern "C" int hilberta_backward(const void *dout, const void *q, const void *k,
                                  void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (p->dtype != HILBERTA_BF16 || p->head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
+    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = (uintptr_t)lse & 3 ? 15 : 0;

@@ -1,5 +1,5 @@
-"""bf16 tensor-core forward with head dim 64 (one 64-column slab per tile) against the oracle,
-including the fused entry / exit gathers and the host-buffer entry point."""
+"""bf16 tensor-core forward and backward with head dim 64 (one 64-column slab per tile) against the
+oracle, including the fused entry / exit gathers and the host-buffer entry point."""
 import numpy as np
 import pytest
 import torch
@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
     (1, 1, 1, 0, 0, 0, 1, 1),
     (64, 64, 1024, 512, 8, 512, 1, 2),
 ])
-def test_head_dim_64_forward(H, W, tile, o, hs, nt, B, heads):
+def test_head_dim_64_forward_and_backward(H, W, tile, o, hs, nt, B, heads):
     S = nt + H * W
     g = torch.Generator().manual_seed(640 + H)
     q, k, v = (torch.randn((B, heads, S, 64), generator=g).bfloat16() for _ in range(3))
@@ -52,10 +52,22 @@ def test_head_dim_64_forward(H, W, tile, o, hs, nt, B, heads):
         plan.forward_host(qh, kh, vh, oh)
         assert plan.status() == 0
         assert torch.equal(oh.view(torch.int16), od.cpu().view(torch.int16))
-        # no backward pass for this head dim
-        bufs = [torch.zeros_like(qp) for _ in range(3)]
-        rc = hb.lib().hilberta_backward(op.data_ptr(), qp.data_ptr(), kp.data_ptr(), vp.data_ptr(), op.data_ptr(),
-                                        lse.data_ptr(), *(t.data_ptr() for t in bufs), plan._h, None)
-        assert rc == hb.ERR_UNSUPPORTED
+        # backward pass on the same plan
+        g2 = torch.Generator().manual_seed(641)
+        do = torch.randn((B, heads, S, 64), generator=g2).bfloat16()
+        ref_g = attn_c.attention_backward(q.float().numpy(), k.float().numpy(), v.float().numpy(),
+                                          do.float().numpy(), ig, grp)
+        dop = do[:, :, p2o].contiguous().cuda()
+        plan.bind_like(qp)
+        grads = [torch.full_like(qp, float("nan")) for _ in range(3)]
+        plan.backward(dop, qp, kp, vp, op, lse, *grads)
+        assert plan.status() == 0
+        for name, t, r in zip(("dq", "dk", "dv"), grads, ref_g):
+            full = torch.empty((B, heads, S, 64), dtype=torch.float64)
+            full[:, :, p2o] = t.cpu().double()
+            assert np.isfinite(full.numpy()).all(), name
+            if np.abs(r).max() > 0:
+                assert orc.rel_l2_err(full.numpy(), r) <= 5e-3, (name, orc.rel_l2_err(full.numpy(), r))
+            assert orc.max_abs_err(full.numpy(), r) <= 1e-2 * max(1.0, np.abs(r).max()), name
     finally:
         plan.destroy()
