@@ -678,25 +678,6 @@ int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, 
 
 namespace {
 
-void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, const int *seg_start,
-               const int *seg_len) {
-    for (int r = 0; r < rows; r += ITEM_ROWS) {
-        WorkItem it{};
-        it.q_start = row0 + r;
-        it.q_rows = std::min(ITEM_ROWS, rows - r);
-        it.n_seg = 0;
-        it.kv_blocks = 0;
-        for (int s = 0; s < n_seg; ++s) {
-            if (seg_len[s] <= 0) continue;
-            it.seg_start[it.n_seg] = seg_start[s];
-            it.seg_len[it.n_seg] = seg_len[s];
-            it.kv_blocks += (seg_len[s] + BN - 1) / BN;
-            ++it.n_seg;
-        }
-        items.push_back(it);
-    }
-}
-
 }  // namespace
 
 int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
@@ -705,63 +686,16 @@ int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
     return HILBERTA_OK;
 }
 
-// Static schedule: every (item, batch*head) unit goes to the least-loaded CTA, longest units
-// first (cost = tile-blocks + a fixed per-unit overhead); units are stored grouped by CTA.
-static int upload_schedule(const std::vector<WorkItem> &items, int bh, int sm_count, WorkUnit **d_units,
-                           int **d_cta_begin, int *n_cta_out) {
-    const long long n_units = (long long)items.size() * bh;
-    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
-    const int n_cta = (int)std::min<long long>(n_units, sm_count);
-    std::vector<std::vector<WorkUnit>> bins(n_cta);
-    typedef std::pair<long long, int> Load;  // (load, cta)
-    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
-    for (int i = 0; i < (int)items.size(); ++i) {
-        // a unit with one query tile has no second tile to overlap its softmax with the MMAs: its
-        // blocks take about 1.3 x half the time of a two-tile unit's (in tenths of a tile-block)
-        const long long cost = (long long)items[i].kv_blocks * (items[i].q_rows > BM ? 20 : 13) + 20;
-        for (int j = 0; j < bh; ++j) {
-            Load top = heap.top();
-            heap.pop();
-            bins[top.second].push_back(WorkUnit{i, j});
-            heap.push(Load(top.first + cost, top.second));
-        }
-    }
-    std::vector<WorkUnit> units;
-    std::vector<int> cta_begin(n_cta + 1, 0);
-    units.reserve((size_t)n_units);
-    for (int c = 0; c < n_cta; ++c) {
-        cta_begin[c] = (int)units.size();
-        units.insert(units.end(), bins[c].begin(), bins[c].end());
-    }
-    cta_begin[n_cta] = (int)units.size();
-    *n_cta_out = n_cta;
-    HB_CUDA(cudaMalloc(d_units, sizeof(WorkUnit) * units.size()));
-    HB_CUDA(cudaMemcpy(*d_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
-    HB_CUDA(cudaMalloc(d_cta_begin, sizeof(int) * cta_begin.size()));
-    HB_CUDA(cudaMemcpy(*d_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
-    return HILBERTA_OK;
-}
-
-// Work list: prefix rows read the whole sequence; the rows of each slid tile
-// read the prefix and the tile's own one or two ranges.  Longest items first.
+// Work list (items of two query tiles, key blocks of 128) and the static schedules.
 int attn_bf16_prepare(hilberta_plan_t *p) {
-    std::vector<WorkItem> items;
-    {
-        const int st[1] = {0}, ln[1] = {p->S};
-        add_items(items, 0, p->P, 1, st, ln);
-    }
-    for (const Window &w : p->h_windows) {
-        const int st[3] = {0, w.seg0_start, w.seg1_start};
-        const int ln[3] = {p->P, w.seg0_len, w.seg1_len};
-        if (w.seg0_len > 0) add_items(items, w.seg0_start, w.seg0_len, 3, st, ln);
-        if (w.seg1_len > 0) add_items(items, w.seg1_start, w.seg1_len, 3, st, ln);
-    }
-    std::stable_sort(items.begin(), items.end(), [](const WorkItem &a, const WorkItem &b) {
-        const long long ca = (long long)a.kv_blocks * (a.q_rows > BM ? 20 : 13);
-        const long long cb = (long long)b.kv_blocks * (b.q_rows > BM ? 20 : 13);
-        return ca > cb;
-    });
+    // a unit with one query tile has no second tile to overlap its softmax with the MMAs: its
+    // blocks take about 1.3 x half the time of a two-tile unit's (costs in tenths of a tile-block)
+    auto cost_of = [](const WorkItem &it) { return (long long)it.kv_blocks * (it.q_rows > BM ? 20 : 13) + 20; };
+    std::vector<WorkItem> items = build_work_items(p, ITEM_ROWS, BN);
+    std::stable_sort(items.begin(), items.end(),
+                     [&](const WorkItem &a, const WorkItem &b) { return cost_of(a) > cost_of(b); });
+    std::vector<long long> cost;
+    for (const WorkItem &it : items) cost.push_back(cost_of(it));
     cudaFree(p->d_work);
     cudaFree(p->d_units);
     cudaFree(p->d_cta_begin);
@@ -779,7 +713,7 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
 
     HB_CUDA(cudaMalloc(&p->d_work, sizeof(WorkItem) * items.size()));
     HB_CUDA(cudaMemcpy(p->d_work, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
-    int rc = upload_schedule(items, p->batch * p->heads, p->sm_count, &p->d_units, &p->d_cta_begin, &p->n_cta);
+    int rc = upload_schedule(items, cost, p->batch * p->heads, p->sm_count, &p->d_units, &p->d_cta_begin, &p->n_cta);
     if (rc != HILBERTA_OK) return rc;
     // slice of heads for the pipelined host-buffer path: the divisor of `heads` nearest to a quarter
     p->chunk_heads = p->heads;
@@ -789,7 +723,7 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
             break;
         }
     if (p->chunk_heads < p->heads) {
-        rc = upload_schedule(items, p->batch * p->chunk_heads, p->sm_count, &p->d_units_chunk, &p->d_cta_begin_chunk,
+        rc = upload_schedule(items, cost, p->batch * p->chunk_heads, p->sm_count, &p->d_units_chunk, &p->d_cta_begin_chunk,
                              &p->n_cta_chunk);
         if (rc != HILBERTA_OK) return rc;
     }

@@ -564,44 +564,17 @@ delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__rest
     }
 }
 
-void add_items(std::vector<WorkItem> &items, int row0, int rows, int n_seg, const int *seg_start,
-               const int *seg_len) {
-    for (int r = 0; r < rows; r += BM) {
-        WorkItem it{};
-        it.q_start = row0 + r;
-        it.q_rows = std::min(BM, rows - r);
-        it.n_seg = 0;
-        it.kv_blocks = 0;
-        for (int s = 0; s < n_seg; ++s) {
-            if (seg_len[s] <= 0) continue;
-            it.seg_start[it.n_seg] = seg_start[s];
-            it.seg_len[it.n_seg] = seg_len[s];
-            it.kv_blocks += (seg_len[s] + BK - 1) / BK;
-            ++it.n_seg;
-        }
-        items.push_back(it);
-    }
-}
-
 }  // namespace
 
 // Work list of the backward kernels: 128 resident rows per item, the rows they exchange
 // gradients with listed as up to three contiguous ranges and counted in blocks of 128.
 // Also allocates the per-row scratch: lse * log2 e for every row, then delta for every row.  Called from hilberta_plan_bind for bf16 bindings.
 int attn_bwd_prepare(hilberta_plan_t *p) {
-    std::vector<WorkItem> items;
-    {
-        const int st[1] = {0}, ln[1] = {p->S};
-        add_items(items, 0, p->P, 1, st, ln);
-    }
-    for (const Window &w : p->h_windows) {
-        const int st[3] = {0, w.seg0_start, w.seg1_start};
-        const int ln[3] = {p->P, w.seg0_len, w.seg1_len};
-        if (w.seg0_len > 0) add_items(items, w.seg0_start, w.seg0_len, 3, st, ln);
-        if (w.seg1_len > 0) add_items(items, w.seg1_start, w.seg1_len, 3, st, ln);
-    }
+    std::vector<WorkItem> items = build_work_items(p, BM, BK);
     std::stable_sort(items.begin(), items.end(),
                      [](const WorkItem &a, const WorkItem &b) { return a.kv_blocks > b.kv_blocks; });
+    std::vector<long long> cost;
+    for (const WorkItem &it : items) cost.push_back((long long)it.kv_blocks + 3);
     cudaFree(p->d_bwd_work);
     cudaFree(p->d_bwd_units);
     cudaFree(p->d_bwd_cta_begin);
@@ -615,37 +588,10 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
     if (items.empty()) return HILBERTA_OK;
 
     const int bh = p->batch * p->heads;
-    const long long n_units = (long long)items.size() * bh;
-    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
-    const int n_cta = (int)std::min<long long>(n_units, p->sm_count);
-    std::vector<std::vector<WorkUnit>> bins(n_cta);
-    typedef std::pair<long long, int> Load;
-    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
-    for (int i = 0; i < (int)items.size(); ++i) {
-        const long long cost = (long long)items[i].kv_blocks + 3;
-        for (int j = 0; j < bh; ++j) {
-            Load top = heap.top();
-            heap.pop();
-            bins[top.second].push_back(WorkUnit{i, j});
-            heap.push(Load(top.first + cost, top.second));
-        }
-    }
-    std::vector<WorkUnit> units;
-    std::vector<int> cta_begin(n_cta + 1, 0);
-    units.reserve((size_t)n_units);
-    for (int c = 0; c < n_cta; ++c) {
-        cta_begin[c] = (int)units.size();
-        units.insert(units.end(), bins[c].begin(), bins[c].end());
-    }
-    cta_begin[n_cta] = (int)units.size();
-    p->n_bwd_cta = n_cta;
     HB_CUDA(cudaMalloc(&p->d_bwd_work, sizeof(WorkItem) * items.size()));
     HB_CUDA(cudaMemcpy(p->d_bwd_work, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
-    HB_CUDA(cudaMalloc(&p->d_bwd_units, sizeof(WorkUnit) * units.size()));
-    HB_CUDA(cudaMemcpy(p->d_bwd_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
-    HB_CUDA(cudaMalloc(&p->d_bwd_cta_begin, sizeof(int) * cta_begin.size()));
-    HB_CUDA(cudaMemcpy(p->d_bwd_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
+    const int rc = upload_schedule(items, cost, bh, p->sm_count, &p->d_bwd_units, &p->d_bwd_cta_begin, &p->n_bwd_cta);
+    if (rc != HILBERTA_OK) return rc;
     HB_CUDA(cudaMalloc(&p->d_delta, sizeof(float) * 2 * (size_t)bh * p->S));
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;

@@ -121,6 +121,11 @@ int launch_attn_fp32(const hilberta_plan_t *p, const void *q, const void *k, con
                      float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk = -1);
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
                      float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk = -1);
+// schedule.cu: work lists (runs of item_rows rows with their up to three key ranges, counted in
+// blocks of `block` rows) and the static longest-first assignment of (item, batch * head) units to CTAs
+std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, int block);
+int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
+                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out);
 int attn_bf16_prepare(hilberta_plan_t *p);
 int attn_bwd_prepare(hilberta_plan_t *p);
 // dq, dk, dv (bf16, physical order, the bound strides) from dout, q, k, v, out and the forward's lse.

@@ -1,0 +1,90 @@
+// Host-side work lists and static schedules shared by the tensor-core kernels.
+//
+// A work item is a run of consecutive physical rows that share one list of up to three
+// contiguous ranges (prefix, tile range, wrapped tile range -- or the whole sequence for
+// prefix rows).  The forward kernel keeps the rows resident as queries and streams the
+// ranges as keys; the backward kernels use the same lists in both directions, because the
+// mask is symmetric (Sec. 3.2 / 3.3).  Every (item, batch * head) unit is assigned to a CTA on
+// the host, longest units first onto the least-loaded CTA, and stored grouped by CTA.
+#include <algorithm>
+#include <functional>
+#include <queue>
+#include <utility>
+
+#include "common.cuh"
+
+namespace hilberta {
+
+static void add_items(std::vector<WorkItem> &items, int row0, int rows, int item_rows, int block, int n_seg,
+                      const int *seg_start, const int *seg_len) {
+    for (int r = 0; r < rows; r += item_rows) {
+        WorkItem it{};
+        it.q_start = row0 + r;
+        it.q_rows = std::min(item_rows, rows - r);
+        it.n_seg = 0;
+        it.kv_blocks = 0;
+        for (int s = 0; s < n_seg; ++s) {
+            if (seg_len[s] <= 0) continue;
+            it.seg_start[it.n_seg] = seg_start[s];
+            it.seg_len[it.n_seg] = seg_len[s];
+            it.kv_blocks += (seg_len[s] + block - 1) / block;
+            ++it.n_seg;
+        }
+        items.push_back(it);
+    }
+}
+
+// Prefix rows see the whole sequence; the rows of each slid tile see the prefix and the
+// tile's own one or two ranges.  item_rows: resident rows per item; block: streamed rows per
+// block (kv_blocks counts them).
+std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, int block) {
+    std::vector<WorkItem> items;
+    {
+        const int st[1] = {0}, ln[1] = {p->S};
+        add_items(items, 0, p->P, item_rows, block, 1, st, ln);
+    }
+    for (const Window &w : p->h_windows) {
+        const int st[3] = {0, w.seg0_start, w.seg1_start};
+        const int ln[3] = {p->P, w.seg0_len, w.seg1_len};
+        if (w.seg0_len > 0) add_items(items, w.seg0_start, w.seg0_len, item_rows, block, 3, st, ln);
+        if (w.seg1_len > 0) add_items(items, w.seg1_start, w.seg1_len, item_rows, block, 3, st, ln);
+    }
+    return items;
+}
+
+// items must be sorted by descending cost.  On success *d_units holds items.size() * bh units
+// grouped by CTA and *d_cta_begin the n_cta + 1 offsets (both device memory, owned by the caller).
+int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
+                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out) {
+    const long long n_units = (long long)items.size() * bh;
+    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    const int n_cta = (int)std::min<long long>(n_units, sm_count);
+    std::vector<std::vector<WorkUnit>> bins(n_cta);
+    typedef std::pair<long long, int> Load;  // (load, cta)
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
+    for (int i = 0; i < (int)items.size(); ++i) {
+        for (int j = 0; j < bh; ++j) {
+            Load top = heap.top();
+            heap.pop();
+            bins[top.second].push_back(WorkUnit{i, j});
+            heap.push(Load(top.first + cost[i], top.second));
+        }
+    }
+    std::vector<WorkUnit> units;
+    std::vector<int> cta_begin(n_cta + 1, 0);
+    units.reserve((size_t)n_units);
+    for (int c = 0; c < n_cta; ++c) {
+        cta_begin[c] = (int)units.size();
+        units.insert(units.end(), bins[c].begin(), bins[c].end());
+    }
+    cta_begin[n_cta] = (int)units.size();
+    *n_cta_out = n_cta;
+    HB_CUDA(cudaMalloc(d_units, sizeof(WorkUnit) * units.size()));
+    HB_CUDA(cudaMemcpy(*d_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
+    HB_CUDA(cudaMalloc(d_cta_begin, sizeof(int) * cta_begin.size()));
+    HB_CUDA(cudaMemcpy(*d_cta_begin, cta_begin.data(), sizeof(int) * cta_begin.size(), cudaMemcpyHostToDevice));
+    return HILBERTA_OK;
+}
+
+}  // namespace hilberta
