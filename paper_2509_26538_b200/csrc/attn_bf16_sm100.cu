@@ -258,30 +258,32 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                 const int nb = item_blocks(wi, seg);
                 for (int j = 0; ok && j < nb; ++j) {
-                    // the K and the V tile of a block share their rows; the table entries are
-                    // requested before the wait for a free slot
+                    // the K and the V tile of a block share their rows: one pass copies both; the
+                    // table entries are requested before the wait for the two free slots
                     int ia, ib;
                     load_rows(wi.seg_start[seg] + j * BN, ia, ib);
-                    for (int kv = 0; kv < 2; ++kv, ++kvc) {
-                        const uint32_t s = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
-#ifdef HB_TIMING
-                        const long long tg0 = clock64();
-#endif
-                        ok = wait_or_abort(bar(KV_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x112);
-                        if (!ok) break;
-#ifdef HB_TIMING
-                        const long long tg1 = clock64();
-#endif
-                        copy_tile(sKV + s * TILE_BYTES, (kv ? prm.gv : prm.gk) + bh_off, ia, ib);
-                        publish(bar(KV_FULL + s));
-#ifdef HB_TIMING
-                        if (tid == 10 * 32) {
-                            atomicAdd(prm.status + 24, (int)((tg1 - tg0) >> 4));
-                            atomicAdd(prm.status + 25, (int)((clock64() - tg1) >> 4));
-                            atomicAdd(prm.status + 26, 1);
+                    const uint32_t sk = kvc % NSTAGE, phk = (kvc / NSTAGE) & 1;
+                    const uint32_t sv = (kvc + 1) % NSTAGE, phv = ((kvc + 1) / NSTAGE) & 1;
+                    kvc += 2;
+                    ok = wait_or_abort(bar(KV_EMPTY + sk), phk ^ 1, &abort_flag, prm.status, 0x112);
+                    if (!ok) break;
+                    ok = wait_or_abort(bar(KV_EMPTY + sv), phv ^ 1, &abort_flag, prm.status, 0x113);
+                    if (!ok) break;
+                    {
+                        // one pass over the rows for both tiles: a shuffle and an address per row pair
+                        const __nv_bfloat16 *k0 = prm.gk + bh_off + chunk * 8, *v0 = prm.gv + bh_off + chunk * 8;
+                        const uint32_t dk0 = sKV + sk * TILE_BYTES + dst_lane, dv0 = sKV + sv * TILE_BYTES + dst_lane;
+#pragma unroll
+                        for (int i = 0; i < 64 / RPI; ++i) {
+                            const int orow = __shfl_sync(0xffffffffu, RPI * i < 32 ? ia : ib, ((RPI * i) & 31) + sub);
+                            const uint32_t o = i * (RPI * 128) + ((c7 ^ ((RPI * i) & 7)) << 4);
+                            const long long so = (long long)max(orow, 0) * prm.stride_s;
+                            cp_async16(dk0 + o, k0 + so, orow >= 0 ? 16 : 0);
+                            cp_async16(dv0 + o, v0 + so, orow >= 0 ? 16 : 0);
                         }
-#endif
                     }
+                    publish(bar(KV_FULL + sk));
+                    publish(bar(KV_FULL + sv));
                 }
             }
         }
