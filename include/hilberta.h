@@ -186,8 +186,8 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  *     delta_i = sum_d dout[i, d] * out[i, d],       dS = P * (dP - delta),
  *     dq = scale * dS k,    dk = scale * dS^T q,    dv = P^T dout.
  *
- * dout, q, k, v, out : device pointers, PHYSICAL order, bf16, the bound shape and
- *                      strides; `out` and `lse` are what hilberta_forward_lse wrote
+ * dout, q, k, v, out : device pointers, PHYSICAL order, the bound dtype, shape and
+ *                      strides (bf16: tensor-core kernels; fp32: plain-FMA kernels); `out` and `lse` are what hilberta_forward_lse wrote
  *                      for these q, k, v.
  * lse                : device pointer, [batch * heads, S] fp32 (natural log).
  * dq, dk, dv         : device pointers, written; same shape and strides as q; must
@@ -199,8 +199,7 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  * the same plan must not overlap on the device.
  *
  * Errors: ERR_INVALID (NULL, misaligned or aliasing pointers, wrong device),
- * ERR_UNBOUND, ERR_UNSUPPORTED (fp32 binding: only the bf16 tensor-core path has a
- * backward pass), ERR_CUDA. */
+ * ERR_UNBOUND, ERR_CUDA. */
 int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                       const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
                       void *stream);

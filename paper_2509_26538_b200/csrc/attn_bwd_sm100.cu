@@ -608,6 +608,8 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
 int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, const void *k, const void *v,
                     const void *out, const float *lse, void *dq, void *dk, void *dv, float *delta,
                     cudaStream_t stream) {
+    if (p->dtype == HILBERTA_FP32)
+        return launch_attn_fp32_bwd(p, dout, q, k, v, out, lse, dq, dk, dv, delta, stream);
     if (p->n_bwd_work == 0) return HILBERTA_OK;
     CUtensorMap mq, mk, mv, mdo;
     int rc;
@@ -696,7 +698,6 @@ extern "C" int hilberta_backward_static(const void *dout, const void *q, const v
                                         const hilberta_plan_t *p, void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = ((uintptr_t)lse & 3) ? 15 : 0;

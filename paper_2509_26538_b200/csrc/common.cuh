@@ -132,5 +132,8 @@ int attn_bwd_prepare(hilberta_plan_t *p);
 int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, const void *k, const void *v,
                     const void *out, const float *lse, void *dq, void *dk, void *dv, float *delta,
                     cudaStream_t stream);
+int launch_attn_fp32_bwd(const hilberta_plan_t *p, const void *dout, const void *q, const void *k, const void *v,
+                         const void *out, const float *lse, void *dq, void *dk, void *dv, float *delta,
+                         cudaStream_t stream);
 int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream);
 }  // namespace hilberta

@@ -562,6 +562,12 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
         rc = attn_bwd_prepare(p);
         if (rc != HILBERTA_OK) return rc;
     }
+    if (dtype == HILBERTA_FP32) {
+        // scratch of the backward pass (delta per row; sized like the bf16 path's)
+        cudaFree(p->d_delta);
+        p->d_delta = nullptr;
+        HB_CUDA(cudaMalloc(&p->d_delta, sizeof(float) * 2 * (size_t)batch * heads * p->S));
+    }
     p->bound = true;
     return HILBERTA_OK;
 }
@@ -609,7 +615,6 @@ extern "C" int hilberta_backward(const void *dout, const void *q, const void *k,
                                  void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (p->dtype != HILBERTA_BF16) return HILBERTA_ERR_UNSUPPORTED;
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = (uintptr_t)lse & 3 ? 15 : 0;

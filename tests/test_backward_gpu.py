@@ -109,9 +109,6 @@ def test_backward_argument_checks():
         assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), ptr[1], ptr[6], ptr[7], plan._h, None) == hb.ERR_INVALID
         assert L.hilberta_backward(ptr[0] + 2, *ptr[1:5], lse.data_ptr(), *ptr[5:8], plan._h, None) == hb.ERR_INVALID
         assert plan.status() == 0
-        f = torch.zeros((1, 1, 256, 64), device="cuda", dtype=torch.float32)
-        plan.bind_like(f)
-        assert L.hilberta_backward(*ptr[:5], lse.data_ptr(), *ptr[5:8], plan._h, None) == hb.ERR_UNSUPPORTED
     finally:
         plan.destroy()
 
@@ -189,5 +186,42 @@ def test_backward_strided_tensors():
         for a, b in ((out, outc), (dq, dqc), (dk, dkc), (dv, dvc)):
             assert torch.equal(a.contiguous().view(torch.int16), b.view(torch.int16))
         assert torch.equal(lse, lsec)
+    finally:
+        plan.destroy()
+
+
+@pytest.mark.parametrize("H,W,tile,o,hs,nt,B,heads,D", [
+    (16, 16, 64, 16, 2, 0, 1, 2, 64),      # the tiny fp32 configuration
+    (16, 16, 64, 48, 2, 5, 2, 2, 32),
+    (12, 20, 64, 9, 2, 7, 1, 1, 128),
+])
+def test_backward_fp32_inputs(H, W, tile, o, hs, nt, B, heads, D):
+    """fp32 bindings take the plain-FMA backward kernels; bar as for the fp32 forward (1e-5 relative
+    to the gradient's scale)."""
+    S = nt + H * W
+    g = torch.Generator().manual_seed(9)
+    q, k, v, do = (torch.randn((B, heads, S, D), generator=g) for _ in range(4))
+    ig, grp = orc.token_classes(H, W, tile, o, hs, nt)
+    ref = attn_c.attention_backward(q.numpy(), k.numpy(), v.numpy(), do.numpy(), ig, grp)
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    try:
+        p2o = torch.from_numpy(plan.export(hb.EXPORT_PHYS2ORIG).astype(np.int64))
+        qp, kp, vp, dop = (t[:, :, p2o].contiguous().cuda() for t in (q, k, v, do))
+        out = torch.empty_like(qp)
+        lse = torch.empty((B, heads, S), device="cuda", dtype=torch.float32)
+        plan.bind_like(qp)
+        plan.forward_lse(qp, kp, vp, out, lse)
+        grads = [torch.full_like(qp, float("nan")) for _ in range(3)]
+        plan.backward(dop, qp, kp, vp, out, lse, *grads)
+        static = [torch.full_like(qp, float("nan")) for _ in range(3)]
+        plan.backward_static(dop, qp, kp, vp, out, lse, *static)
+        assert plan.status() == 0
+        for name, t, t2, r in zip(("dq", "dk", "dv"), grads, static, ref):
+            assert torch.equal(t, t2), name
+            full = torch.empty((B, heads, S, D), dtype=torch.float64)
+            full[:, :, p2o] = t.cpu().double()
+            scale = max(1.0, np.abs(r).max())
+            assert orc.max_abs_err(full.numpy(), r) <= 1e-5 * scale, (name, orc.max_abs_err(full.numpy(), r))
+            assert orc.rel_l2_err(full.numpy(), r) <= 1e-5, (name, orc.rel_l2_err(full.numpy(), r))
     finally:
         plan.destroy()
