@@ -27,6 +27,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 NOMINAL_BF16_TFLOPS = 2250.0
+L2_BYTES = 126 * 2**20   # B200 L2
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one forward launch, from the
 # ncu capture summarised in profiles/attn_bf16_kernel_flux2048.md (555.1 MB read + 92.4 MB written).
@@ -183,7 +184,9 @@ def workload_config(wl, n_gpus):
                         f"{wl.shared_region}, offset {wl.layer_offset}",
             "S": wl.S, "tile": wl.tile, "shared_region": wl.shared_region, "layer_offset": wl.layer_offset,
             "step": "permute(Q,K,V) + sparse forward with the exit unpermute fused into its epilogue",
-            "l2": "inputs larger than L2 (Q+K+V+O = %d MB)" % (4 * wl.batch * wl.heads * wl.S * wl.head_dim * 2 // 2**20),
+            "l2": ("inputs larger than L2 (Q+K+V+O = %d MB)" if 4 * wl.batch * wl.heads * wl.S * wl.head_dim * 2 > L2_BYTES
+                   else "Q+K+V+O = %d MB fits in L2: the steps rotate through several copies of their buffers") %
+                  (4 * wl.batch * wl.heads * wl.S * wl.head_dim * 2 // 2**20),
             "parallelism": f"replicas x{n_gpus} (independent batches, no collective)"}
 
 
@@ -251,6 +254,13 @@ def main():
     q, k, v = make_qkv(wl.with_(seed=wl.seed + 100 * rank))
     qd, kd, vd = (t.cuda() for t in (q, k, v))
     qp, kp, vp, op, od = (torch.empty_like(qd) for _ in range(5))
+    # Workloads whose tensors fit in L2 (126 MB) rotate through several copies of the step's
+    # buffers, so that no step finds its inputs cached by the previous one.
+    step_bytes = 7 * qd.numel() * qd.element_size()      # q, k, v, their permuted copies, out
+    n_sets = 1 if step_bytes >= 2 * L2_BYTES else min(8, -(-3 * L2_BYTES // step_bytes))
+    sets = [(qd, kd, vd, qp, kp, vp, od)]
+    for _ in range(n_sets - 1):
+        sets.append(tuple(t.clone() for t in sets[0]))
 
     t0 = time.perf_counter()
     plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text, groups=args.groups)
@@ -263,20 +273,21 @@ def main():
 
     stream = torch.cuda.current_stream()
 
-    def step(ev=None):
+    def step(ev=None, i=0):
+        a_q, a_k, a_v, a_qp, a_kp, a_vp, a_o = sets[i % n_sets]
         if ev:
             ev[0].record(stream)
-        plan.permute(qd, qp)
-        plan.permute(kd, kp)
-        plan.permute(vd, vp)
+        plan.permute(a_q, a_qp)
+        plan.permute(a_k, a_kp)
+        plan.permute(a_v, a_vp)
         if ev:
             ev[1].record(stream)
-        plan.forward_unpermute(qp, kp, vp, od)   # exit gather fused into the epilogue
+        plan.forward_unpermute(a_qp, a_kp, a_vp, a_o)   # exit gather fused into the epilogue
         if ev:
             ev[2].record(stream)
 
-    for _ in range(args.warmup):
-        step()
+    for i in range(args.warmup):
+        step(None, i)
     torch.cuda.synchronize()
     assert plan.status() == 0, "device-side wait timed out"
 
@@ -290,7 +301,7 @@ def main():
     sampler.start()
     start.record(stream)
     for i in range(args.steps):
-        step(evs[i])
+        step(evs[i], args.warmup + i)
     stop.record(stream)
     torch.cuda.synchronize()
     if distributed:
@@ -391,9 +402,10 @@ def main():
         torch.cuda.synchronize()
         n_f = max(5, min(args.steps, 30))
         fev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_f)]
-        for a, b_ in fev:
+        for i, (a, b_) in enumerate(fev):
+            f_q, f_k, f_v = sets[i % n_sets][0:3]
             a.record(stream)
-            plan.forward_fused(qd, kd, vd, of, True, True)
+            plan.forward_fused(f_q, f_k, f_v, of, True, True)
             b_.record(stream)
         torch.cuda.synchronize()
         assert plan.status() == 0, "device-side wait timed out"
@@ -454,12 +466,20 @@ def main():
         sched_flops = sum(4.0 * wl.head_dim * wl.heads * wl.batch * int(plans[o].export(hb.EXPORT_NNZ)[0])
                           for o in offs)
 
+        # every layer of a real step has its own activations: the layers rotate through the
+        # permuted copies of the buffer sets, so a layer does not find its Q, K, V in L2
+        for a_q, a_k, a_v, a_qp, a_kp, a_vp, _ in sets[1:]:
+            plan.permute(a_q, a_qp)
+            plan.permute(a_k, a_kp)
+            plan.permute(a_v, a_vp)
+
         def sched_step():
             plan.permute(qd, qp)
             plan.permute(kd, kp)
             plan.permute(vd, vp)
-            for o in offs[:-1]:
-                plans[o].forward(qp, kp, vp, op)
+            for li, o in enumerate(offs[:-1]):
+                lq, lk, lv = sets[li % n_sets][3:6]
+                plans[o].forward(lq, lk, lv, op)
             plans[offs[-1]].forward_unpermute(qp, kp, vp, od)
 
         for _ in range(3):
@@ -476,7 +496,8 @@ def main():
         schedule = {"layers": SCHEDULE_LAYERS, "distinct_plans": len(plans), "ms_per_step": sched_ms,
                     "ms_per_layer": sched_ms / SCHEDULE_LAYERS, "useful_tflops": sched_flops / (sched_ms * 1e-3) / 1e12,
                     "offsets": "(layer * tile / 4) mod HW", "reps": reps,
-                    "note": "same Q/K/V for every layer (synthetic); one entry permute of Q, K, V; the last layer writes in original order"}
+                    "note": "one entry permute of Q, K, V; the layers rotate through %d sets of Q/K/V buffers; "
+                            "the last layer writes in original order" % n_sets}
         for p_ in plans.values():
             assert p_.status() == 0
             p_.destroy()
