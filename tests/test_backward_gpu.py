@@ -225,3 +225,43 @@ def test_backward_fp32_inputs(H, W, tile, o, hs, nt, B, heads, D):
             assert orc.rel_l2_err(full.numpy(), r) <= 1e-5, (name, orc.rel_l2_err(full.numpy(), r))
     finally:
         plan.destroy()
+
+
+@pytest.mark.parametrize("name", ["flux2048", "flux4096"])
+def test_backward_identities_at_full_size(name):
+    """Properties that hold at any size, on the whole bench-shaped problem: shifting every key by one
+    vector changes no softmax weight (sum_j dk_j = 0), every row's weights sum to one
+    (sum_j dv_j = sum_i dO_i), and scaling q up and k down leaves the output unchanged
+    (<q, dq> = <k, dk> per head).  Each is checked against the size of the terms that cancel."""
+    from paper_2509_26538_b200.inputs import WORKLOADS
+    wl = WORKLOADS[name]
+    g = torch.Generator(device="cuda").manual_seed(wl.seed)
+    shape = (wl.batch, wl.heads, wl.S, wl.head_dim)
+    qp, kp, vp, dop = (torch.randn(shape, generator=g, device="cuda").to(torch.bfloat16) for _ in range(4))
+    plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
+    try:
+        plan.bind_like(qp)
+        out = torch.empty_like(qp)
+        lse = torch.empty(shape[:3], device="cuda", dtype=torch.float32)
+        plan.forward_lse(qp, kp, vp, out, lse)
+        dq, dk, dv = (torch.full_like(qp, float("nan")) for _ in range(3))
+        plan.backward(dop, qp, kp, vp, out, lse, dq, dk, dv)
+        assert plan.status() == 0
+        for t in (dq, dk, dv):
+            assert torch.isfinite(t.float()).all()
+        # stored gradients carry bf16 rounding (2^-9 relative each); sums of S such terms are
+        # checked against sqrt(S) * 2^-8 of their root-mean-square size
+        S = wl.S
+        dkf = dk.double()
+        tol_k = (S ** 0.5) * 2.0 ** -8 * dkf.pow(2).mean().sqrt()
+        assert dkf.sum(dim=2).abs().max() <= 4 * tol_k
+        dvf = dv.double()
+        want = dop.double().sum(dim=2)
+        tol_v = (S ** 0.5) * 2.0 ** -8 * max(dvf.pow(2).mean().sqrt(), dop.double().pow(2).mean().sqrt())
+        assert (dvf.sum(dim=2) - want).abs().max() <= 4 * tol_v
+        a = (qp.double() * dq.double()).sum(dim=(2, 3))
+        b = (kp.double() * dkf).sum(dim=(2, 3))
+        size = (qp.double() * dq.double()).abs().sum(dim=(2, 3))
+        assert ((a - b).abs() <= 2.0 ** -6 * size).all()
+    finally:
+        plan.destroy()
