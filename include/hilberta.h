@@ -115,11 +115,18 @@ int hilberta_plan_groups(int H, int W, int groups, int layer_offset, int shared_
  * tokens, original order [text | (f * H + r) * W + c], reordered along a THREE-dimensional
  * Hilbert curve so that a tile is a compact spatio-temporal block; tiles, slide and
  * wrap-around are those of hilberta_plan on that curve.  The paper names the idea and fixes
- * neither the curve nor the shared region; this library uses the curve of Skilling's
- * transpose construction with axes (frame, row, col), starting at cell (0, 0, 0), on the
- * smallest enclosing power-of-two cube (side n >= max(frames, H, W); cells outside the volume
- * are padding, as for general image shapes; `tile` must divide n^3), and a centred shared BOX
- * of shared_frames x shared_region x shared_region cells (both even, both zero for none).
+ * neither the curve nor the shared region; this library's reading: with the frame axis padded
+ * to 2^a >= frames and the image axes to 2^b >= max(H, W),
+ *   a <  b (a clip shorter than a frame is wide, the usual case): the image plane is cut into
+ *          macro cells of 2^a x 2^a pixels visited in the order of the 2-D curve of
+ *          hilberta_plan; the cube of 2^a frames above a macro cell is walked by a 3-D
+ *          Hilbert curve (Skilling's transpose construction, axes (frame, row, col), starting
+ *          at the cube's cell (0, 0, 0)); index = macro index * 8^a + index inside the cube;
+ *          the padded curve has 2^(2b + a) positions;
+ *   a >= b: the whole volume lies in one cube of side 2^a walked by the 3-D curve.
+ * Cells outside the volume are padding, as for general image shapes; `tile` must divide the
+ * padded length.  The shared region is a centred BOX of shared_frames x shared_region x
+ * shared_region cells (both even, both zero for none).
  * frames >= 2; frames, H, W <= 128.  Everything downstream (export, bind, forward,
  * backward, permute) is unchanged: the kernels only ever see contiguous physical ranges. */
 int hilberta_plan_video(int frames, int H, int W, int tile, int layer_offset, int shared_region,

@@ -119,35 +119,70 @@ def hilbert3d_point(d: int, k: int):
 def padded_side(H: int, W: int, frames: int = 1) -> int:
     """Side n = 2^k of the smallest enclosing power-of-two square (Appendix "Hilbert
     Curve for General Shape": the curve is built on an enclosing regular grid and the
-    H x W sub-region is extracted; cells outside it are padding).  With frames > 1
-    the enclosing shape is a cube that also holds the frame axis."""
+    H x W sub-region is extracted; cells outside it are padding).  For a video volume
+    the frame axis is padded separately (video_orders)."""
     if H < 1 or W < 1 or frames < 1:
         raise ValueError("empty grid")
     n = 1
-    while n < max(H, W, frames if frames > 1 else 1):
+    while n < max(H, W):
         n *= 2
+    if frames > 1:
+        a, b = video_orders(H, W, frames)
+        n = 1 << max(a, b)
     return n
 
 
+def video_orders(H: int, W: int, frames: int):
+    """(a, b): the frame axis is padded to 2^a >= frames, the two image axes to 2^b."""
+    a = 1
+    while (1 << a) < frames:
+        a += 1
+    b = 0
+    while (1 << b) < max(H, W):
+        b += 1
+    return a, b
+
+
 def padded_length(H: int, W: int, frames: int = 1) -> int:
-    """Length of the padded curve: n^2 for an image, n^3 for a video volume."""
-    n = padded_side(H, W, frames)
-    return n * n if frames == 1 else n * n * n
+    """Length of the padded curve: n^2 for an image; for a video volume 2^(2b + a) when the clip
+    is shorter than the image is wide (a < b), else the cube (2^a)^3."""
+    if frames == 1:
+        n = padded_side(H, W)
+        return n * n
+    a, b = video_orders(H, W, frames)
+    return 1 << (2 * b + a) if a < b else 1 << (3 * a)
 
 
 def hilbert_cell_index(H: int, W: int, frames: int = 1) -> np.ndarray:
     """row-major cell id r*W + c -> Hilbert index of the cell on the padded n x n grid.
-    int32[HW].  For a power-of-two square this is pi^-1 itself.  With frames > 1:
-    cell id (f*H + r)*W + c -> index on the 3-D curve of the padded cube."""
-    n = padded_side(H, W, frames)
+    int32[HW].  For a power-of-two square this is pi^-1 itself.
+
+    With frames > 1: cell id (f*H + r)*W + c -> index on the spatio-temporal curve (Sec. 5).
+    A clip is usually much shorter than a frame is wide, and one cube around everything would
+    be mostly padding.  So, with the frame axis padded to 2^a and the image axes to 2^b, a < b:
+    the image plane is cut into macro cells of 2^a x 2^a pixels, visited in the order of the 2-D
+    curve of Sec. 3.1 (order b - a); the 2^a x 2^a x 2^a block of cells above a macro cell (all
+    frames) is walked by the 3-D curve.  index = macro index * 8^a + index inside the block.
+    Tiles of a multiple of 8^j positions are then unions of compact spatio-temporal blocks.
+    If a >= b the whole volume sits in one cube of side 2^a walked by the 3-D curve."""
     if frames > 1:
-        k = _log2_exact(n)
+        a, b = video_orders(H, W, frames)
         out = np.empty(frames * H * W, dtype=np.int32)
-        for d in range(n * n * n):
-            f, y, x = hilbert3d_point(d, k)
-            if f < frames and y < H and x < W:
-                out[(f * H + y) * W + x] = d
+        if a >= b:
+            for d in range(1 << (3 * a)):
+                f, y, x = hilbert3d_point(d, a)
+                if f < frames and y < H and x < W:
+                    out[(f * H + y) * W + x] = d
+            return out
+        block = 1 << (3 * a)
+        inner = [hilbert3d_point(d, a) for d in range(block)]
+        for m, (mx, my) in enumerate(hilbert_points(b - a)):        # (x, y) = (col, row) of the macro cell
+            for d, (f, y, x) in enumerate(inner):
+                r, c = (my << a) + y, (mx << a) + x
+                if f < frames and r < H and c < W:
+                    out[(f * H + r) * W + c] = m * block + d
         return out
+    n = padded_side(H, W)
     pts = hilbert_points(_log2_exact(n))
     out = np.empty(H * W, dtype=np.int32)
     for d, (x, y) in enumerate(pts):

@@ -62,6 +62,7 @@ struct hilberta_plan_s {
     int device;
     int H, W, HW, k_log2;   // image grid; padded side n = 2^k_log2 >= max(H, W); HW = number of grid cells
     int frames, shared_frames;  // video volume: frames x H x W cells on a 3-D curve (frames == 1: an image)
+    int ka_log2, kb_log2;       // video: frame axis padded to 2^ka, image axes to 2^kb
     int NP;                 // n * n: length of the padded Hilbert curve the tiles are cut on
     bool compact;           // tiles are equal groups over the non-shared tokens (Algorithm 1) instead of curve intervals
     int tile, offset, shared_region, n_text, n_shared, T, S, P;

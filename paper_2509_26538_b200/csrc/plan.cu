@@ -22,13 +22,8 @@ std::atomic<uint64_t> g_launches{0};
 // ---------------------------------------------------------------------------
 enum : unsigned char { CELL_PAD = 0, CELL_REAL = 1, CELL_SHARED = 2 };
 
-__global__ void hilbert_lut_kernel(int k, int H, int W, int *__restrict__ cell_of_pd,
-                                   int *__restrict__ pd_of_cell, unsigned char *__restrict__ kind_by_pd,
-                                   int sh_r0, int sh_c0, int sh_side) {
+__device__ __forceinline__ int hilbert2d_index(int k, int row, int col) {
     const int n = 1 << k;
-    const int pc = blockIdx.x * blockDim.x + threadIdx.x;   // padded cell
-    if (pc >= n * n) return;
-    const int row = pc >> k, col = pc & (n - 1);
     int x = col, y = row;
     int d = 0;
     for (int s = n >> 1; s > 0; s >>= 1) {
@@ -45,6 +40,17 @@ __global__ void hilbert_lut_kernel(int k, int H, int W, int *__restrict__ cell_o
             y = t;
         }
     }
+    return d;
+}
+
+__global__ void hilbert_lut_kernel(int k, int H, int W, int *__restrict__ cell_of_pd,
+                                   int *__restrict__ pd_of_cell, unsigned char *__restrict__ kind_by_pd,
+                                   int sh_r0, int sh_c0, int sh_side) {
+    const int n = 1 << k;
+    const int pc = blockIdx.x * blockDim.x + threadIdx.x;   // padded cell
+    if (pc >= n * n) return;
+    const int row = pc >> k, col = pc & (n - 1);
+    const int d = hilbert2d_index(k, row, col);
     if (row < H && col < W) {
         const int cell = row * W + col;
         pd_of_cell[cell] = d;
@@ -58,17 +64,16 @@ __global__ void hilbert_lut_kernel(int k, int H, int W, int *__restrict__ cell_o
 }
 
 // Video volumes (Sec. 5, "Extension to Video Diffusion"): one thread per cell of the padded
-// n x n x n cube, axes (frame, row, col).  The cell's index on the 3-D Hilbert curve comes from
-// the coordinate -> index direction of Skilling's transpose construction: per level, from the top
-// bit down, an inversion or an exchange against axis 0; then a Gray encoding across the axes; the
-// index is the bit interleave of the three resulting words (frame word most significant).
-__global__ void hilbert3d_lut_kernel(int k, int F, int H, int W, int *__restrict__ cell_of_pd,
-                                     int *__restrict__ pd_of_cell, unsigned char *__restrict__ kind_by_pd,
-                                     int sh_f0, int sh_r0, int sh_c0, int sh_side, int sh_frames) {
-    const int n = 1 << k;
-    const int pc = blockIdx.x * blockDim.x + threadIdx.x;   // padded cell
-    if (pc >= n * n * n) return;
-    const int f = pc >> (2 * k), row = (pc >> k) & (n - 1), col = pc & (n - 1);
+// volume of 2^a frames by 2^b x 2^b pixels.  A clip is usually much shorter than a frame is wide
+// (a < b): the image plane is cut into macro cells of 2^a x 2^a pixels visited in the order of the
+// 2-D curve, and the 2^a-cube of cells above a macro cell is walked by a 3-D Hilbert curve:
+// index = macro index * 8^a + index inside the cube.  With a >= b the whole volume is one cube of
+// side 2^a.  The 3-D index comes from the coordinate -> index direction of Skilling's transpose
+// construction with axes (frame, row, col): per level, from the top bit down, an inversion or an
+// exchange against axis 0; then a Gray encoding across the axes; the index is the bit interleave
+// of the three resulting words (frame word most significant).
+__device__ __forceinline__ int hilbert3d_index(int k, int f, int row, int col) {
+    if (k == 0) return 0;
     unsigned X0 = f, X1 = row, X2 = col;
     for (unsigned Q = 1u << (k - 1); Q > 1; Q >>= 1) {
         const unsigned Pm = Q - 1;
@@ -99,6 +104,23 @@ __global__ void hilbert3d_lut_kernel(int k, int F, int H, int W, int *__restrict
     int d = 0;
     for (int b = k - 1; b >= 0; --b)
         d = (d << 3) | (int)(((X0 >> b) & 1) << 2 | ((X1 >> b) & 1) << 1 | ((X2 >> b) & 1));
+    return d;
+}
+
+__global__ void hilbert3d_lut_kernel(int a, int b, int F, int H, int W, int *__restrict__ cell_of_pd,
+                                     int *__restrict__ pd_of_cell, unsigned char *__restrict__ kind_by_pd,
+                                     int sh_f0, int sh_r0, int sh_c0, int sh_side, int sh_frames) {
+    const int side = a >= b ? a : b;         // log2 of the padded image side
+    const int pc = blockIdx.x * blockDim.x + threadIdx.x;   // padded cell, frame-major
+    if (pc >= (1 << (a + 2 * side))) return;
+    const int f = pc >> (2 * side), row = (pc >> side) & ((1 << side) - 1), col = pc & ((1 << side) - 1);
+    int d;
+    if (a >= b) {
+        d = hilbert3d_index(a, f, row, col);
+    } else {
+        const int m = (1 << a) - 1;
+        d = (hilbert2d_index(b - a, row >> a, col >> a) << (3 * a)) + hilbert3d_index(a, f, row & m, col & m);
+    }
     if (f < F && row < H && col < W) {
         const int cell = (f * H + row) * W + col;
         pd_of_cell[cell] = d;
@@ -306,7 +328,7 @@ static int build_plan(hilberta_plan_t *p) {
             break;
         }
         if (p->frames > 1)
-            hilbert3d_lut_kernel<<<(NP + 255) / 256, 256>>>(p->k_log2, p->frames, p->H, p->W, d_cell_of_pd,
+            hilbert3d_lut_kernel<<<(NP + 255) / 256, 256>>>(p->ka_log2, p->kb_log2, p->frames, p->H, p->W, d_cell_of_pd,
                                                             d_pd_of_cell, d_kind, p->frames / 2 - p->shared_frames / 2,
                                                             sh_r0, sh_c0, p->shared_region, p->shared_frames);
         else
@@ -394,12 +416,20 @@ static int make_plan(int frames, int H, int W, int tile, int groups, int layer_o
     if (H > 1024 || W > 1024) return HILBERTA_ERR_UNSUPPORTED;
     if (frames > 1 && (H > 128 || W > 128 || frames > 128)) return HILBERTA_ERR_UNSUPPORTED;
     const int HW = frames * H * W;        // grid cells = image (or video) tokens
-    int side = H > W ? H : W;
-    if (frames > 1 && frames > side) side = frames;
-    int k_log2 = 0;                       // padded side n = 2^k >= max(H, W[, frames])
-    while ((1 << k_log2) < side) ++k_log2;
-    if (frames > 1 && k_log2 < 1) k_log2 = 1;
-    const int NP = 1 << ((frames > 1 ? 3 : 2) * k_log2);   // length of the padded curve
+    int k_log2 = 0;                       // padded image side n = 2^k >= max(H, W)
+    while ((1 << k_log2) < (H > W ? H : W)) ++k_log2;
+    int ka = 0, kb = k_log2;              // video: frames padded to 2^ka, image axes to 2^kb
+    int NP = 1 << (2 * k_log2);           // length of the padded curve
+    if (frames > 1) {
+        ka = 1;
+        while ((1 << ka) < frames) ++ka;
+        if (ka >= kb) {                   // one cube of side 2^ka
+            k_log2 = ka;
+            NP = 1 << (3 * ka);
+        } else {                          // macro cells of 2^ka x 2^ka pixels under cubes of side 2^ka
+            NP = 1 << (2 * kb + ka);
+        }
+    }
     if (shared_region % 2 || shared_region > H || shared_region > W) return HILBERTA_ERR_INVALID;
     if (frames > 1) {
         if (shared_frames % 2 || shared_frames > frames) return HILBERTA_ERR_INVALID;
@@ -434,6 +464,8 @@ static int make_plan(int frames, int H, int W, int tile, int groups, int layer_o
     p->HW = HW;
     p->NP = NP;
     p->k_log2 = k_log2;
+    p->ka_log2 = ka;
+    p->kb_log2 = kb;
     p->compact = compact;
     p->tile = tile;
     const long long period = compact ? R : NP;

@@ -37,14 +37,49 @@ def test_order_one_table():
         assert orc.hilbert3d_point(d, 1) == (f, r, c)
 
 
+def _bitpair_d2xy(k, d):
+    """The 2-D curve by the classic iterative index-to-point conversion (not the oracle's recursion)."""
+    x = y = 0
+    t, s = d, 1
+    while s < (1 << k):
+        rx = 1 & (t >> 1)
+        ry = 1 & (t ^ rx)
+        if ry == 0:
+            if rx == 1:
+                x, y = s - 1 - x, s - 1 - y
+            x, y = y, x
+        x += s * rx
+        y += s * ry
+        t >>= 2
+        s <<= 1
+    return x, y
+
+
 def _naive_mask(F, H, W, tile, o, hs, fs, n_text):
-    """The three clauses of the mask tested on grid coordinates, token by token."""
-    n = orc.padded_side(H, W, F)
-    k = n.bit_length() - 1
-    NP = n ** 3
-    index_of = {}
-    for d in range(NP):
-        index_of[orc.hilbert3d_point(d, k)] = d
+    """The three clauses of the mask tested on grid coordinates, token by token; the curve index
+    of a cell is looked up in tables built here: the 3-D curve inside a block of 2^a frames by
+    2^a x 2^a pixels, and (for clips shorter than the image is wide) the 2-D order of the blocks."""
+    a = 1
+    while (1 << a) < F:
+        a += 1
+    b = 0
+    while (1 << b) < max(H, W):
+        b += 1
+    if a >= b:
+        NP = 1 << (3 * a)
+        index_of = {orc.hilbert3d_point(d, a): d for d in range(NP)}
+    else:
+        NP = 1 << (2 * b + a)
+        inner = {orc.hilbert3d_point(d, a): d for d in range(1 << (3 * a))}
+        macro = {}
+        for m in range(1 << (2 * (b - a))):
+            x, y = _bitpair_d2xy(b - a, m)
+            macro[(y, x)] = m
+        index_of = {}
+        for f in range(F):
+            for r in range(H):
+                for c in range(W):
+                    index_of[(f, r, c)] = (macro[(r >> a, c >> a)] << (3 * a)) + inner[(f, r & ((1 << a) - 1), c & ((1 << a) - 1))]
     S = n_text + F * H * W
     f0, r0, c0 = F // 2 - fs // 2, H // 2 - hs // 2, W // 2 - hs // 2
 

@@ -15,9 +15,11 @@ pytestmark = pytest.mark.gpu
     (4, 4, 4, 16, 5, 2, 2, 3),
     (2, 4, 4, 8, 3, 2, 2, 0),
     (3, 4, 2, 16, 7, 0, 0, 2),
-    (8, 16, 16, 512, 200, 4, 2, 77),      # padded to a 16-cube: half the curve is padding
+    (8, 16, 16, 512, 200, 4, 2, 77),      # a clip shorter than the image is wide: 2 x 2 macro cells of 8-cubes
     (16, 16, 16, 256, 64, 8, 4, 0),       # a full cube
     (5, 12, 20, 1024, 999, 2, 2, 9),      # nothing is a power of two
+    (8, 64, 64, 2048, 512, 8, 4, 100),    # a video-shaped volume without any padding
+    (32, 8, 8, 4096, 77, 2, 2, 0),        # more frames than pixels per side: one 32-cube
 ])
 def test_video_plan_bit_exact(F, H, W, tile, o, hs, fs, nt):
     ref = orc.plan_arrays(H, W, tile, o, hs, nt, frames=F, shared_frames=fs)
@@ -31,8 +33,8 @@ def test_video_plan_bit_exact(F, H, W, tile, o, hs, fs, nt):
         assert np.array_equal(plan.export(hb.EXPORT_WINDOWS), ref["windows"])
         assert int(plan.export(hb.EXPORT_NNZ)[0]) == ref["nnz"]
         info = plan.export(hb.EXPORT_INFO).tolist()
-        n = orc.padded_side(H, W, F)
-        assert info == [H, W, tile, o % n ** 3, hs, nt, hs * hs * fs, n ** 3 // tile, n, F, fs]
+        n, NP = orc.padded_side(H, W, F), orc.padded_length(H, W, F)
+        assert info == [H, W, tile, o % NP, hs, nt, hs * hs * fs, NP // tile, n, F, fs]
     finally:
         plan.destroy()
 
@@ -43,6 +45,7 @@ def test_video_plan_argument_checks():
     h = ctypes.c_void_p()
     for args in ((1, 4, 4, 16, 0, 0, 0, 0),        # one frame is an image: use hilberta_plan
                  (4, 4, 4, 24, 0, 0, 0, 0),        # tile does not divide 64
+                 (2, 4, 4, 64, 0, 0, 0, 0),        # the padded curve of a 2 x 4 x 4 clip has 32 positions
                  (4, 4, 4, 16, 0, 2, 0, 0),        # shared square without temporal extent
                  (4, 4, 4, 16, 0, 2, 3, 0),        # odd temporal extent
                  (4, 4, 4, 16, 0, 2, 6, 0)):       # longer than the clip
