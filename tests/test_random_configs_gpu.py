@@ -1,0 +1,98 @@
+"""Seeded random configurations: plan tables bit-exact against the oracle, and forward / backward in
+tolerance on the smaller ones.  Shapes, tiles, offsets, shared regions, text lengths and the three
+plan flavours (curve tiles, equal groups, video volumes) are drawn at random from their valid ranges."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attn_c
+from oracle import hilberta_oracle as orc
+from paper_2509_26538_b200 import binding as hb
+
+pytestmark = pytest.mark.gpu
+
+
+def _divisors(n):
+    return [d for d in range(1, n + 1) if n % d == 0]
+
+
+def _draw(rng):
+    kind = rng.choice(["image", "groups", "video"], p=[0.5, 0.25, 0.25])
+    H, W = int(rng.integers(1, 41)), int(rng.integers(1, 41))
+    F = int(rng.integers(2, 10)) if kind == "video" else 1
+    if kind == "video":
+        H, W = int(rng.integers(1, 17)), int(rng.integers(1, 17))
+    hs = int(rng.choice([0, 0, 2, 4, 6]))
+    hs = min(hs, (min(H, W) // 2) * 2)
+    fs = 0
+    if kind == "video":
+        fs = min(int(rng.choice([2, 4])), (F // 2) * 2) if hs else 0
+        if fs == 0:
+            hs = 0
+    nt = int(rng.choice([0, 0, 1, 7, 33, 130]))
+    NP = orc.padded_length(H, W, F)
+    n_sh = hs * hs * (fs if kind == "video" else 1)
+    cells = F * H * W
+    if kind == "groups":
+        R = cells - n_sh
+        if R < 1:
+            hs, n_sh, R = 0, 0, cells
+        groups = int(rng.choice(_divisors(R)))
+        o = int(rng.integers(0, 3 * R + 1))
+        return dict(kind=kind, H=H, W=W, F=1, tile=0, groups=groups, o=o, hs=hs, fs=0, nt=nt)
+    tile = int(rng.choice(_divisors(NP)))
+    o = int(rng.integers(0, 3 * NP + 1))
+    return dict(kind=kind, H=H, W=W, F=F, tile=tile, groups=0, o=o, hs=hs, fs=fs, nt=nt)
+
+
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_random_configuration(seed):
+    rng = np.random.default_rng(4242 + seed)
+    c = _draw(rng)
+    H, W, F, tile, groups, o, hs, fs, nt = (c[k] for k in ("H", "W", "F", "tile", "groups", "o", "hs", "fs", "nt"))
+    if groups:
+        ref = orc.plan_arrays_compact(H, W, groups, o, hs, nt)
+        ig, grp = orc.token_classes_compact(H, W, groups, o, hs, nt)
+    else:
+        ref = orc.plan_arrays(H, W, tile, o, hs, nt, frames=F, shared_frames=fs)
+        ig, grp = orc.token_classes(H, W, tile, o, hs, nt, frames=F, shared_frames=fs)
+    plan = hb.Plan(H, W, tile, o, hs, nt, groups=groups, frames=F, shared_frames=fs)
+    try:
+        for key, sel in (("hil_d2t", hb.EXPORT_HIL_D2T), ("hil_t2d", hb.EXPORT_HIL_T2D),
+                         ("phys2orig", hb.EXPORT_PHYS2ORIG), ("orig2phys", hb.EXPORT_ORIG2PHYS),
+                         ("shared_runs", hb.EXPORT_SHARED_RUNS), ("windows", hb.EXPORT_WINDOWS)):
+            assert np.array_equal(plan.export(sel), ref[key]), (c, key)
+        assert int(plan.export(hb.EXPORT_NNZ)[0]) == ref["nnz"], c
+        S = nt + F * H * W
+        if S > 1400:
+            return
+        g = torch.Generator().manual_seed(seed)
+        heads = int(rng.integers(1, 3))
+        q, k, v, do = (torch.randn((1, heads, S, 128), generator=g).to(torch.bfloat16) for _ in range(4))
+        f32 = lambda t: t.float().numpy()
+        ref_o = attn_c.attention_rows(f32(q), f32(k), f32(v), ig, grp)
+        ref_g = attn_c.attention_backward(f32(q), f32(k), f32(v), f32(do), ig, grp)
+        qd, kd, vd = (t.cuda() for t in (q, k, v))
+        plan.bind_like(qd)
+        out = torch.full_like(qd, float("nan"))
+        plan.forward_fused(qd, kd, vd, out, in_original=True, out_original=True)
+        p2o = torch.from_numpy(ref["phys2orig"].astype(np.int64))
+        qp, kp, vp, dop = (t[:, :, p2o].contiguous().cuda() for t in (q, k, v, do))
+        outp = torch.empty_like(qp)
+        lse = torch.empty((1, heads, S), device="cuda", dtype=torch.float32)
+        plan.forward_lse(qp, kp, vp, outp, lse)
+        grads = [torch.full_like(qp, float("nan")) for _ in range(3)]
+        plan.backward(dop, qp, kp, vp, outp, lse, *grads)
+        assert plan.status() == 0, c
+        got = out.cpu().double().numpy()
+        assert np.isfinite(got).all(), c
+        assert orc.max_abs_err(got, ref_o) <= 1e-2 and orc.rel_l2_err(got, ref_o) <= 5e-3, c
+        for t, r in zip(grads, ref_g):
+            full = torch.empty((1, heads, S, 128), dtype=torch.float64)
+            full[:, :, p2o] = t.cpu().double()
+            assert np.isfinite(full.numpy()).all(), c
+            if np.abs(r).max() > 0:
+                assert orc.rel_l2_err(full.numpy(), r) <= 5e-3, c
+            assert orc.max_abs_err(full.numpy(), r) <= 1e-2 * max(1.0, np.abs(r).max()), c
+    finally:
+        plan.destroy()
