@@ -1,6 +1,6 @@
-/* hilberta.h -- C ABI of the HilbertA sparse-attention forward for NVIDIA B200 (sm_100a).
+/* hilberta.h -- C ABI of HilbertA sparse attention (forward and backward) for NVIDIA B200 (sm_100a).
  *
- * The library implements the inference hot path of Hilbert-curve tiled sparse
+ * The library implements the hot path of Hilbert-curve tiled sparse
  * attention for diffusion transformers: tokens of an H x W image grid are
  * reordered along a Hilbert curve (Sec. 3.1), the reordered sequence is cut
  * into tiles of N_T tokens with dense attention inside each tile, the tile
@@ -47,12 +47,12 @@ extern "C" {
 /* status codes */
 #define HILBERTA_OK 0
 #define HILBERTA_ERR_INVALID (-1)     /* bad argument value */
-#define HILBERTA_ERR_UNSUPPORTED (-2) /* valid in the method, not built (non-square / non power-of-two grid, head_dim) */
+#define HILBERTA_ERR_UNSUPPORTED (-2) /* valid in the method, not built (grid or volume too large, head_dim) */
 #define HILBERTA_ERR_ARCH (-3)        /* current device is not compute capability 10.x */
 #define HILBERTA_ERR_CUDA (-4)        /* a CUDA call failed; see hilberta_last_cuda_error() */
 #define HILBERTA_ERR_NOMEM (-5)       /* host or device allocation failed */
-#define HILBERTA_ERR_BUFFER (-6)      /* export buffer too small; *needed is set */
-#define HILBERTA_ERR_UNBOUND (-7)     /* hilberta_forward before hilberta_plan_bind */
+#define HILBERTA_ERR_BUFFER (-6)      /* export buffer too small (*needed is set), or problem too large for a fixed scratch array */
+#define HILBERTA_ERR_UNBOUND (-7)     /* an attention call before hilberta_plan_bind */
 #define HILBERTA_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired (see hilberta_plan_status) */
 
 /* element types */
