@@ -58,6 +58,13 @@ extern "C" {
 /* element types */
 #define HILBERTA_BF16 0
 #define HILBERTA_FP32 1
+/* q, k, v are e4m3 bytes (4 exponent bits, 3 mantissa bits, bias 7, no infinities; the "fn"
+ * encoding); out is bf16.  Forward only.  The paper's kernel computes in 16-bit types (Sec. 4.1);
+ * this is the same Algorithm 1 with 8-bit tensor-core operands: the softmax weights are rounded to
+ * e4m3 as well before they multiply V, accumulation and the softmax itself stay fp32.  Any
+ * per-tensor quantisation scales are the caller's: fold those of q and k into `scale`, multiply
+ * v's into `out`. */
+#define HILBERTA_FP8_E4M3 2
 
 /* selectors for hilberta_plan_export */
 #define HILBERTA_EXPORT_HIL_D2T 0     /* int32[HW]   Hilbert rank (curve order among the real cells) -> cell r*W+c */
@@ -147,13 +154,18 @@ int hilberta_plan_export(const hilberta_plan_t *plan, int what, void *host_buf, 
  * configuration line: batch Z, heads, head dim D, softmax scale s, strides).
  *
  *   batch, heads   >= 1.  The same mask serves every (batch, head).
- *   head_dim       bf16: 128 or 64.  fp32: 32, 64 or 128.  Others: ERR_UNSUPPORTED.
- *   dtype          HILBERTA_BF16 (tensor-core kernel) or HILBERTA_FP32 (plain FMA kernel).
+ *   head_dim       bf16: 128 or 64.  fp32: 32, 64 or 128.  e4m3: 128.  Others: ERR_UNSUPPORTED.
+ *   dtype          HILBERTA_BF16 (tensor-core kernel), HILBERTA_FP32 (plain FMA kernel) or
+ *                  HILBERTA_FP8_E4M3 (tensor-core kernel, 8-bit operands, bf16 output; forward,
+ *                  forward_lse, forward_unpermute and forward_fused only -- hilberta_backward*
+ *                  and hilberta_forward_host return ERR_UNSUPPORTED).
  *   stride_b, stride_h, stride_s
  *                  element strides of q, k, v and out (all four share them) for
  *                  the batch, head and token axes; the head_dim axis is contiguous.
  *                  0 for all three means the dense [batch, heads, S, head_dim] layout.
- *                  bf16 needs every stride to be a multiple of 8 elements (16 bytes).
+ *                  bf16 needs every stride to be a multiple of 8 elements (16 bytes);
+ *                  e4m3 a multiple of 16 elements (q, k, v are then 16-byte aligned row
+ *                  by row, and so is the bf16 `out`, which uses the same element strides).
  *   scale          softmax scale s; <= 0 selects 1/sqrt(head_dim).
  *
  * Builds the kernel's work list (device memory) and may allocate and synchronise.
@@ -167,7 +179,7 @@ int hilberta_plan_bind(hilberta_plan_t *plan, int batch, int heads, int head_dim
  *
  *   q, k, v   device pointers, PHYSICAL token order, layout as bound; read only.
  *   out       device pointer, same layout, written; must not overlap q, k or v.
- *             bf16: all four 16-byte aligned.
+ *             bf16 and e4m3: all four 16-byte aligned.
  *   plan      a bound plan.
  *   stream    the launch is asynchronous on this stream; no allocation, no
  *             synchronisation.

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libhilberta.so")
 OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_ARCH, ERR_CUDA, ERR_NOMEM, ERR_BUFFER, ERR_UNBOUND, ERR_TIMEOUT = (
     -1, -2, -3, -4, -5, -6, -7, -8)
-BF16, FP32 = 0, 1
+BF16, FP32, FP8_E4M3 = 0, 1, 2
 (EXPORT_HIL_D2T, EXPORT_HIL_T2D, EXPORT_PHYS2ORIG, EXPORT_ORIG2PHYS, EXPORT_SHARED_RUNS, EXPORT_WINDOWS,
  EXPORT_NNZ, EXPORT_INFO) = range(8)
 
@@ -114,6 +114,8 @@ def _dtype_code(t) -> int:
         return BF16
     if t.dtype == torch.float32:
         return FP32
+    if t.dtype == torch.float8_e4m3fn:
+        return FP8_E4M3
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 

@@ -29,6 +29,7 @@
 #include <functional>
 #include <mutex>
 #include <queue>
+#include <type_traits>
 #include <utility>
 
 #include "common.cuh"
@@ -45,12 +46,18 @@ constexpr int QT = 2;          // query tiles per work item
 constexpr int ITEM_ROWS = QT * BM;
 constexpr int NSTAGE = 5;      // K/V ring slots (K0 V0 K1 V1 ...)
 constexpr int SLAB_BYTES = BN * 128;     // one 64-column slab of 128 rows (128-byte swizzled rows)
-// head dim HD = 128: a tile is two slabs (32 KB); HD = 64: one slab (16 KB)
-__host__ __device__ constexpr int tile_bytes(int hd) { return BN * hd * 2; }
+// bf16, head dim HD = 128: a tile is two slabs (32 KB); HD = 64: one slab (16 KB).
+// e4m3 (fp8 = true), HD = 128: rows of 128 bytes, one slab.
+__host__ __device__ constexpr int tile_bytes(int hd, bool fp8 = false) { return BN * hd * (fp8 ? 1 : 2); }
 constexpr int THREADS = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle (register donors)
-__host__ __device__ constexpr int smem_bytes(int hd) { return (QT + NSTAGE) * tile_bytes(hd) + 1024; }
+__host__ __device__ constexpr int smem_bytes(int hd, bool fp8 = false) { return (QT + NSTAGE) * tile_bytes(hd, fp8) + 1024; }
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
+// e4m3 weights: the running maximum may lag by 2^4 and every weight carries a factor 2^4 (divided
+// out with the row sum at the end), so weights lie in (0, 2^8] under e4m3's largest value 448 and
+// the smallest nonzero one, 2^-9, is 2^-13 of the reference maximum.
+constexpr float RESCALE_THRESHOLD_FP8 = 4.0f;
+constexpr float P_SHIFT_FP8 = 4.0f;
 #ifndef HB_POLY_MASK
 #define HB_POLY_MASK 3   // pair i of every 16 runs its two exponentials on the FMA pipes when (i & MASK) == MASK (3: one pair in four); 0xff = never
 #endif
@@ -93,7 +100,7 @@ struct KernelParams : Params {};
 template <>
 struct KernelParams<true> : Params {
     const int *in_map;
-    const __nv_bfloat16 *gq, *gk, *gv;
+    const void *gq, *gk, *gv;
 };
 
 __device__ __forceinline__ int item_blocks(const WorkItem &it, int seg) {
@@ -125,30 +132,46 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
     return p;
 }
 
-// S_t = Q_t K^T for one 128-key block: 8 MMAs of K = 16.
-template <int HD>
+// S_t = Q_t K^T for one 128-key block: HD / 16 MMAs of K = 16 (bf16) or HD / 32 of K = 32 (e4m3);
+// either way an MMA consumes 32 bytes of every row.
+template <int HD, bool FP8>
 __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t sQt, uint32_t sKslot) {
-    constexpr uint32_t IDESC = idesc_bf16_f32(BM, BN, 0, 0);
     // the start-address field is the low 14 bits (16-byte units): stepping K is one add
     const uint64_t dq = smem_desc_sw128(sQt, 16, 1024), dk = smem_desc_sw128(sKslot, 16, 1024);
+    if constexpr (FP8) {
+        constexpr uint32_t IDESC = idesc_e4m3_f32(BM, BN, 0);
 #pragma unroll
-    for (int k = 0; k < HD / 16; ++k) {
-        const uint64_t off = (uint64_t)(((k >> 2) * SLAB_BYTES + (k & 3) * 32) >> 4);
-        mma_ss(tmem_s, dq + off, dk + off, IDESC, k > 0);
+        for (int k = 0; k < HD / 32; ++k) mma_ss_f8(tmem_s, dq + (uint64_t)((k * 32) >> 4), dk + (uint64_t)((k * 32) >> 4), IDESC, k > 0);
+    } else {
+        constexpr uint32_t IDESC = idesc_bf16_f32(BM, BN, 0, 0);
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+            const uint64_t off = (uint64_t)(((k >> 2) * SLAB_BYTES + (k & 3) * 32) >> 4);
+            mma_ss(tmem_s, dq + off, dk + off, IDESC, k > 0);
+        }
     }
 }
 
 // O_t (+)= P_t V for one 128-key block: P from TMEM, V row-major in smem (N-major operand).
-// `half` selects keys [64 half, +64) of the block: four MMAs of K = 16.
-template <int HD>
+// `half` selects keys [64 half, +64) of the block: four MMAs of K = 16 (bf16: 8 columns of P and
+// 16 rows of V each) or two of K = 32 (e4m3: 8 columns of P, four weights per column, and 32 rows of V).
+template <int HD, bool FP8>
 __device__ __forceinline__ void issue_pv_half(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, int half,
                                               bool accumulate) {
-    constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
     const uint64_t dv = smem_desc_sw128(sVslot + half * 8192, SLAB_BYTES, 1024);
+    if constexpr (FP8) {
+        constexpr uint32_t IDESC = idesc_e4m3_f32(BM, HD, 1);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        mma_ts(tmem_o, tmem_p + half * 32 + k * 8, dv + (uint64_t)((k * 2048) >> 4), IDESC,
-               (accumulate || k > 0) ? 1u : 0u);
+        for (int k = 0; k < 2; ++k)
+            mma_ts_f8(tmem_o, tmem_p + half * 16 + k * 8, dv + (uint64_t)((k * 4096) >> 4), IDESC,
+                      (accumulate || k > 0) ? 1u : 0u);
+    } else {
+        constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            mma_ts(tmem_o, tmem_p + half * 32 + k * 8, dv + (uint64_t)((k * 2048) >> 4), IDESC,
+                   (accumulate || k > 0) ? 1u : 0u);
+        }
     }
 }
 
@@ -162,7 +185,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int sr
 // GATHER = true : the tensors are in ORIGINAL order (the entry gather of Sec. 3.4 fused in): two loader
 // warps fetch every tile row through the permutation table with 16-byte cp.async copies and place it
 // where a 128-byte-swizzled TMA box would have put it, so everything downstream is unchanged.
-template <bool GATHER, int HD>
+// FP8: q, k, v hold e4m3 bytes (HD = 128 only); the weights P are rounded to e4m3 as well; out stays bf16.
+template <bool GATHER, int HD, bool FP8 = false>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const KernelParams<GATHER> prm) {
@@ -170,8 +194,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __shared__ uint64_t bars[NUM_BARS];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    constexpr int TILE_BYTES = tile_bytes(HD);
-    constexpr int NSLAB = HD / 64;
+    static_assert(!FP8 || HD == 128, "e4m3 operands: head dim 128 only");
+    constexpr int TILE_BYTES = tile_bytes(HD, FP8);
+    constexpr int NSLAB = TILE_BYTES / SLAB_BYTES;
+    using elem_t = typename std::conditional<FP8, uint8_t, __nv_bfloat16>::type;
+    constexpr int EPC = 16 / (int)sizeof(elem_t);   // elements per 16-byte chunk
 
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sQ = smem_u32(smem);
@@ -221,7 +248,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         // instruction (16 bytes per lane; a row is CH = HD / 8 lanes wide).  Lane L fetches the
         // table entries of rows L and 32 + L of that range once per tile; the lanes that copy a
         // row pick its entry up by shuffle, so the table costs one load latency per tile.
-        constexpr int CH = HD / 8, RPI = 32 / CH;
+        constexpr int CH = HD / EPC, RPI = 32 / CH;
         const int lane = tid & 31, chunk = lane % CH, sub = lane / CH, wrow = (warp - 10) * 64;
         const uint32_t dst_lane = (uint32_t)((chunk >> 3) * SLAB_BYTES + (wrow + sub) * 128);
         const int c7 = (chunk & 7) ^ sub;   // row & 7 = (RPI i + sub) & 7 = ((RPI i) & 7) ^ sub
@@ -230,8 +257,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             ia = pa < prm.S ? __ldg(prm.in_map + pa) : -1;   // rows beyond the sequence are
             ib = pb < prm.S ? __ldg(prm.in_map + pb) : -1;   // zero-filled, as TMA does
         };
-        auto copy_tile = [&](uint32_t dst_tile, const __nv_bfloat16 *base, int ia, int ib) {
-            const __nv_bfloat16 *src0 = base + chunk * 8;
+        auto copy_tile = [&](uint32_t dst_tile, const elem_t *base, int ia, int ib) {
+            const elem_t *src0 = base + chunk * EPC;
             const uint32_t dst0 = dst_tile + dst_lane;
 #pragma unroll
             for (int i = 0; i < 64 / RPI; ++i) {
@@ -252,7 +279,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int t = 0; t < nt; ++t) {
                 int ia, ib;
                 load_rows(wi.q_start + t * BM, ia, ib);
-                copy_tile(sQ + t * TILE_BYTES, prm.gq + bh_off, ia, ib);
+                copy_tile(sQ + t * TILE_BYTES, (const elem_t *)prm.gq + bh_off, ia, ib);
             }
             publish(bar(Q_FULL));
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
@@ -271,7 +298,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (!ok) break;
                     {
                         // one pass over the rows for both tiles: a shuffle and an address per row pair
-                        const __nv_bfloat16 *k0 = prm.gk + bh_off + chunk * 8, *v0 = prm.gv + bh_off + chunk * 8;
+                        const elem_t *k0 = (const elem_t *)prm.gk + bh_off + chunk * EPC;
+                        const elem_t *v0 = (const elem_t *)prm.gv + bh_off + chunk * EPC;
                         const uint32_t dk0 = sKV + sk * TILE_BYTES + dst_lane, dv0 = sKV + sv * TILE_BYTES + dst_lane;
 #pragma unroll
                         for (int i = 0; i < 64 / RPI; ++i) {
@@ -368,7 +396,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t) {
-                    issue_qk<HD>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
+                    issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
                     mma_commit(bar(S_FULL + t));
                 }
                 mma_commit(bar(KV_EMPTY + slot_of(2 * g)));
@@ -400,7 +428,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef HB_TIMING
                         tm_p += clock64() - tp0;
 #endif
-                        issue_pv_half<HD>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
+                        issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
 #ifdef HB_TIMING
                         const long long tp1 = clock64();
 #endif
@@ -411,10 +439,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         tm_p += clock64() - tp1;
 #endif
                         tc_fence_after();
-                        issue_pv_half<HD>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
+                        issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
                         mma_commit(bar(PV_DONE + t));
                         if (more) {
-                            issue_qk<HD>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
+                            issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
                             mma_commit(bar(S_FULL + t));
                         }
                     }
@@ -458,6 +486,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const int bh = unit.bh;
             const int b = bh / prm.heads, h = bh % prm.heads;
             float m_ref = 0.f, l = 0.f;
+            float l_fix = 0.f;   // e4m3 only: rounding error of every block's largest weight (kept out of lse)
             bool first = true;
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                 const int nb = item_blocks(wi, seg);
@@ -493,7 +522,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     if (first) {
                         m_ref = mx;
                         first = false;
-                    } else if (__any_sync(0xffffffffu, mx > m_ref + RESCALE_THRESHOLD)) {
+                    } else if (__any_sync(0xffffffffu, mx > m_ref + (FP8 ? RESCALE_THRESHOLD_FP8 : RESCALE_THRESHOLD))) {
                         // the accumulator of the blocks so far belongs to the old reference
                         ok = wait_or_abort(bar(PV_DONE + t), (cPV - 1) & 1, &abort_flag, prm.status, 0x303 + t);
                         if (!ok) break;
@@ -502,6 +531,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         const float alpha = ex2(m_ref - m_new);
                         m_ref = m_new;
                         l *= alpha;
+                        if constexpr (FP8) l_fix *= alpha;
 #pragma unroll
                         for (int c = 0; c < HD / 32; ++c) {
                             uint32_t o[32];
@@ -512,13 +542,17 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                             tmem_st32(tO + c * 32, o);
                         }
                     }
-                    const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_ref, -m_ref);
+                    const float nm = FP8 ? P_SHIFT_FP8 - m_ref : -m_ref;
+                    const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(nm, nm);
                     float2 sum[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
                     // The row sum is taken over the fp32 weights; the P V MMA sees them rounded
                     // to bf16.  For the block's largest weight -- the one that dominates a
                     // near-one-hot row -- the rounding error is added to the sum, so numerator
                     // and denominator round together where it matters.
-                    {
+                    if constexpr (FP8) {
+                        const float pm = ex2(mx + nm);
+                        l_fix += round_e4m3(pm) - pm;
+                    } else {
                         const float pm = ex2(mx - m_ref);
                         l += __uint_as_float(pack_bf16(0.f, pm) & 0xffff0000u) - pm;
                     }
@@ -538,10 +572,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                 p.x = ex2(x.x);
                                 p.y = ex2(x.y);
                             }
-                            pk[i] = pack_bf16(p.x, p.y);
+                            if constexpr (FP8) {
+                                // four weights per column: pairs 2 i' and 2 i' + 1 share pk[i']
+                                const uint32_t h = pack_e4m3x2(p.x, p.y);
+                                if (i & 1) pk[i >> 1] |= h << 16;
+                                else pk[i >> 1] = h;
+                            } else {
+                                pk[i] = pack_bf16(p.x, p.y);
+                            }
                             sum[i & 3] = __fadd2_rn(sum[i & 3], p);
                         }
-                        tmem_st16(tS + c * 16, pk);
+                        if constexpr (FP8) tmem_st8(tS + c * 8, pk);
+                        else tmem_st16(tS + c * 16, pk);
                         if (HB_SPLIT_P ? (c & 1) : (c == 3)) {  // keys [64 (c >> 1), +64) are in TMEM
                             tmem_wait_st();
                             tc_fence_before();
@@ -567,7 +609,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             ok = wait_or_abort(bar(PV_DONE + t), (cPV - 1) & 1, &abort_flag, prm.status, 0x305 + t);
             if (!ok) break;
             tc_fence_after();
-            const float inv = 1.f / l;
+            const float inv = 1.f / (FP8 ? l + l_fix : l);
             const int row = t * BM + r;
             // each thread stores its own row, so writing it at its ORIGINAL position instead
             // of the physical one (the exit gather of Sec. 3.4 fused in) costs one index read
@@ -577,7 +619,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                   (long long)out_row * prm.stride_s;
             // m_ref and l are in the base-2 domain of the scaled logits: LSE = ln 2 * (m_ref + log2 l)
             if (prm.lse && row < wi.q_rows)
-                prm.lse[(long long)bh * prm.S + out_row] = 0.6931471805599453f * (m_ref + log2f(l));
+                prm.lse[(long long)bh * prm.S + out_row] =
+                    0.6931471805599453f * (m_ref - (FP8 ? P_SHIFT_FP8 : 0.f) + log2f(l));
 #pragma unroll
             for (int c = 0; c < HD / 32; ++c) {
                 uint32_t o[32];
@@ -659,16 +702,20 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
-// [batch, heads, S, 128] bf16 with element strides -> 4-D map, box = 64 columns x box_rows rows.
+// [batch, heads, S, head_dim] with element strides -> 4-D map, box = 128 bytes of a row (64 bf16 or
+// 128 e4m3 columns) x box_rows rows.
 int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, int box_rows, int heads) {
     if (heads <= 0) heads = p->heads;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return HILBERTA_ERR_CUDA;
+    const bool fp8 = p->dtype == HILBERTA_FP8_E4M3;
+    const cuuint64_t esz = fp8 ? 1 : 2;
     cuuint64_t dims[4] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->S, (cuuint64_t)heads, (cuuint64_t)p->batch};
-    cuuint64_t strides[3] = {(cuuint64_t)p->stride_s * 2, (cuuint64_t)p->stride_h * 2, (cuuint64_t)p->stride_b * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    cuuint64_t strides[3] = {(cuuint64_t)p->stride_s * esz, (cuuint64_t)p->stride_h * esz, (cuuint64_t)p->stride_b * esz};
+    cuuint32_t box[4] = {fp8 ? 128u : 64u, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+    CUresult r = enc(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+                     const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -742,6 +789,12 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             smem_bytes(64));
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            smem_bytes(128, true));
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            smem_bytes(128, true));
     });
     HB_CUDA(attr_err);
     return HILBERTA_OK;
@@ -753,9 +806,10 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     int heads = p->heads, n_cta = p->n_cta;
     const WorkUnit *units = p->d_units;
     const int *cta_begin = p->d_cta_begin;
+    const bool fp8 = p->dtype == HILBERTA_FP8_E4M3;
     if (chunk >= 0 && p->chunk_heads < p->heads) {
         // a slice of heads: same strides, shifted base pointers, the slice's own schedule
-        if (lse) return HILBERTA_ERR_INVALID;
+        if (lse || fp8) return HILBERTA_ERR_INVALID;
         heads = p->chunk_heads;
         const long long off = (long long)chunk * heads * p->stride_h;
         q = (const __nv_bfloat16 *)q + off;
@@ -790,17 +844,21 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
         KernelParams<true> gprm;
         static_cast<Params &>(gprm) = prm;
         gprm.in_map = in_map;
-        gprm.gq = (const __nv_bfloat16 *)q;
-        gprm.gk = (const __nv_bfloat16 *)k;
-        gprm.gv = (const __nv_bfloat16 *)v;
-        if (p->head_dim == 128)
+        gprm.gq = q;
+        gprm.gk = k;
+        gprm.gv = v;
+        if (fp8)
+            attn_bf16_kernel<true, 128, true><<<n_cta, THREADS, smem_bytes(128, true), stream>>>(mq, mk, mv, gprm);
+        else if (p->head_dim == 128)
             attn_bf16_kernel<true, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, gprm);
         else
             attn_bf16_kernel<true, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, gprm);
     } else {
         KernelParams<false> pprm;
         static_cast<Params &>(pprm) = prm;
-        if (p->head_dim == 128)
+        if (fp8)
+            attn_bf16_kernel<false, 128, true><<<n_cta, THREADS, smem_bytes(128, true), stream>>>(mq, mk, mv, pprm);
+        else if (p->head_dim == 128)
             attn_bf16_kernel<false, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, pprm);
         else
             attn_bf16_kernel<false, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, pprm);

@@ -608,6 +608,7 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
 int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, const void *k, const void *v,
                     const void *out, const float *lse, void *dq, void *dk, void *dv, float *delta,
                     cudaStream_t stream) {
+    if (p->dtype == HILBERTA_FP8_E4M3) return HILBERTA_ERR_UNSUPPORTED;  // e4m3 bindings are forward only
     if (p->dtype == HILBERTA_FP32)
         return launch_attn_fp32_bwd(p, dout, q, k, v, out, lse, dq, dk, dv, delta, stream);
     if (p->n_bwd_work == 0) return HILBERTA_OK;

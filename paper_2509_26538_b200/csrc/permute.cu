@@ -41,11 +41,11 @@ row_gather_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, const 
 static int gather(const void *src, void *dst, const int *index, const hilberta_plan_t *p, int batch,
                   int row_elems, int dtype, cudaStream_t stream) {
     if (!p || !src || !dst || batch < 1 || row_elems < 1) return HILBERTA_ERR_INVALID;
-    if (dtype != HILBERTA_BF16 && dtype != HILBERTA_FP32) return HILBERTA_ERR_INVALID;
+    if (dtype != HILBERTA_BF16 && dtype != HILBERTA_FP32 && dtype != HILBERTA_FP8_E4M3) return HILBERTA_ERR_INVALID;
     int dev = -1;
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;  // the plan's tables live on another device
-    const size_t esz = dtype == HILBERTA_BF16 ? 2 : 4;
+    const size_t esz = dtype == HILBERTA_BF16 ? 2 : dtype == HILBERTA_FP8_E4M3 ? 1 : 4;
     const size_t row_bytes = (size_t)row_elems * esz;
     if (row_bytes % 16 || ((uintptr_t)src & 15) || ((uintptr_t)dst & 15)) return HILBERTA_ERR_INVALID;
     const size_t bytes = row_bytes * (size_t)p->S * (size_t)batch;

@@ -567,8 +567,9 @@ extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *ho
 extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int head_dim, int dtype,
                                   int64_t stride_b, int64_t stride_h, int64_t stride_s, float scale) {
     if (!p || batch < 1 || heads < 1 || head_dim < 1) return HILBERTA_ERR_INVALID;
-    if (dtype != HILBERTA_BF16 && dtype != HILBERTA_FP32) return HILBERTA_ERR_INVALID;
+    if (dtype != HILBERTA_BF16 && dtype != HILBERTA_FP32 && dtype != HILBERTA_FP8_E4M3) return HILBERTA_ERR_INVALID;
     if (dtype == HILBERTA_BF16 && head_dim != 128 && head_dim != 64) return HILBERTA_ERR_UNSUPPORTED;
+    if (dtype == HILBERTA_FP8_E4M3 && head_dim != 128) return HILBERTA_ERR_UNSUPPORTED;
     if (dtype == HILBERTA_FP32 && head_dim != 32 && head_dim != 64 && head_dim != 128)
         return HILBERTA_ERR_UNSUPPORTED;
     if (stride_b == 0 && stride_h == 0 && stride_s == 0) {
@@ -578,6 +579,7 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
     }
     if (stride_b <= 0 || stride_h <= 0 || stride_s < head_dim) return HILBERTA_ERR_INVALID;
     if (dtype == HILBERTA_BF16 && ((stride_b | stride_h | stride_s) & 7)) return HILBERTA_ERR_INVALID;
+    if (dtype == HILBERTA_FP8_E4M3 && ((stride_b | stride_h | stride_s) & 15)) return HILBERTA_ERR_INVALID;
     if ((int64_t)batch * heads > 65535) return HILBERTA_ERR_INVALID;
     p->bound = false;
     p->batch = batch;
@@ -592,6 +594,11 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
         int rc = attn_bf16_prepare(p);
         if (rc != HILBERTA_OK) return rc;
         rc = attn_bwd_prepare(p);
+        if (rc != HILBERTA_OK) return rc;
+    }
+    if (dtype == HILBERTA_FP8_E4M3) {
+        // forward only: the bf16 kernel's work list and schedule, no backward tables
+        int rc = attn_bf16_prepare(p);
         if (rc != HILBERTA_OK) return rc;
     }
     if (dtype == HILBERTA_FP32) {
@@ -680,6 +687,7 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
     int dev = -1;
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;
+    if (p->dtype == HILBERTA_FP8_E4M3) return HILBERTA_ERR_UNSUPPORTED;  // input and output element sizes differ
     const size_t esz = p->dtype == HILBERTA_BF16 ? 2 : 4;
     const size_t bytes = (size_t)p->batch * p->heads * p->S * p->head_dim * esz;
     const size_t slot = (bytes + 255) & ~(size_t)255;

@@ -23,7 +23,7 @@ class Workload:
     batch: int
     heads: int
     head_dim: int
-    dtype: str  # "bf16" or "fp32"
+    dtype: str  # "bf16", "fp32" or "fp8" (e4m3 q, k, v; bf16 out)
     tile: int
     shared_region: int
     layer_offset: int
@@ -62,7 +62,7 @@ def schedule_offset(layer: int, tile: int, HW: int) -> int:
 
 
 def torch_dtype(name: str) -> torch.dtype:
-    return {"bf16": torch.bfloat16, "fp32": torch.float32}[name]
+    return {"bf16": torch.bfloat16, "fp32": torch.float32, "fp8": torch.float8_e4m3fn}[name]
 
 
 def make_qkv(wl: Workload, heads: int | None = None, q_gain: float = 1.0):
