@@ -207,6 +207,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the dense / SDPA context rows")
     ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass row")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the e4m3-operand forward row")
     ap.add_argument("--schedule", action="store_true",
                     help="also time the 57-layer per-step schedule (one permute, 57 forwards with the "
                          "per-layer offsets, one unpermute) on the chosen workload's shape")
@@ -455,6 +456,35 @@ def main():
         }
         del dop, grads, lse
 
+    # ---- the same forward with e4m3 operands (not part of the metric): q, k, v rounded to 8-bit floats
+    fp8 = None
+    if world == 1 and not args.no_fp8 and wl.dtype == "bf16" and wl.head_dim == 128 and not args.groups:
+        f8 = torch.float8_e4m3fn
+        f_sets = [tuple(t.to(f8) for t in s_[3:6]) for s_ in sets]
+        plan8 = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
+        plan8.bind_like(f_sets[0][0])
+        o8 = torch.empty_like(op)
+        for i in range(3):
+            plan8.forward(*f_sets[i % n_sets], o8)
+        torch.cuda.synchronize()
+        n_8 = max(5, min(args.steps, 30))
+        fev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_8)]
+        for i, (a, b_) in enumerate(fev):
+            a.record(stream)
+            plan8.forward(*f_sets[i % n_sets], o8)
+            b_.record(stream)
+        torch.cuda.synchronize()
+        assert plan8.status() == 0, "device-side wait timed out"
+        assert torch.isfinite(o8.float()).all()
+        ms8 = sorted(a.elapsed_time(b_) for a, b_ in fev)
+        m8 = ms8[len(ms8) // 2]
+        fp8 = {"ms_per_call_median": m8, "ms_per_call_min": ms8[0], "useful_tflops": flops / (m8 * 1e-3) / 1e12,
+               "speedup_vs_bf16_forward": statistics.median(fwd_ms) / m8,
+               "note": "q, k, v and the softmax weights in e4m3 (kind::f8f6f4 MMAs), fp32 softmax and accumulation, "
+                       "bf16 output; tolerance rel-L2 4e-2 (weights have three mantissa bits)"}
+        plan8.destroy()
+        del f_sets, o8
+
     schedule = None
     if args.schedule:
         from paper_2509_26538_b200.inputs import SCHEDULE_LAYERS, schedule_offset
@@ -528,7 +558,7 @@ def main():
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_source": peaks["source"] + " burst",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "traffic": FORWARD_DRAM_TRAFFIC_BYTES.get(wl.name)},
-        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "fused_step": fused, "backward": backward, "schedule57": schedule,
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "fused_step": fused, "backward": backward, "fp8_forward": fp8, "schedule57": schedule,
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
                              "(4.36 ms per call at 2048^2, 16 tiles)", "same_gpu": context_rows},
     }

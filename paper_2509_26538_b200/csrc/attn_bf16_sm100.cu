@@ -61,6 +61,15 @@ constexpr float P_SHIFT_FP8 = 4.0f;
 #ifndef HB_POLY_MASK
 #define HB_POLY_MASK 3   // pair i of every 16 runs its two exponentials on the FMA pipes when (i & MASK) == MASK (3: one pair in four); 0xff = never
 #endif
+#ifndef HB_POLY_MASK_FP8
+#define HB_POLY_MASK_FP8 HB_POLY_MASK
+#endif
+#ifndef HB_POLY_DEG_FP8
+#define HB_POLY_DEG_FP8 2
+#endif
+#ifndef HB_POLY_DEG
+#define HB_POLY_DEG 3
+#endif
 #ifndef HB_SPLIT_P
 #define HB_SPLIT_P 1     // hand P to the MMA issuer in two halves
 #endif
@@ -118,15 +127,22 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // bits), f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.8e-5, far below bf16
 // rounding), 2^n by an exponent add.  Used for a fixed share of the exponentials so that
 // the MUFU unit and the FMA pipes split the work.  x is clamped at -126 (result ~0).
+template <int DEG = 3>
 __device__ __forceinline__ float2 ex2_poly2(float2 x) {
     x.x = fmaxf(x.x, -126.f);
     x.y = fmaxf(x.y, -126.f);
     const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
     const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
     const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-    float2 p = __ffma2_rn(f, make_float2(0.055088773f, 0.055088773f), make_float2(0.24260406f, 0.24260406f));
-    p = __ffma2_rn(p, f, make_float2(0.69327623f, 0.69327623f));
-    p = __ffma2_rn(p, f, make_float2(0.99992895f, 0.99992895f));
+    float2 p;
+    if constexpr (DEG == 2) {
+        p = __ffma2_rn(f, make_float2(0.23842697f, 0.23842697f), make_float2(0.7034453f, 0.7034453f));
+        p = __ffma2_rn(p, f, make_float2(1.00044307f, 1.00044307f));
+    } else {
+        p = __ffma2_rn(f, make_float2(0.055088773f, 0.055088773f), make_float2(0.24260406f, 0.24260406f));
+        p = __ffma2_rn(p, f, make_float2(0.69327623f, 0.69327623f));
+        p = __ffma2_rn(p, f, make_float2(0.99992895f, 0.99992895f));
+    }
     p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
     p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
     return p;
@@ -566,8 +582,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                                                     __uint_as_float(s[c * 32 + 2 * i + 1])),
                                                         sc2, nm2);
                             float2 p;
-                            if ((i & HB_POLY_MASK) == HB_POLY_MASK) {
-                                p = ex2_poly2(x);  // a fixed share of the pairs runs on the FMA pipes
+                            constexpr int PM = FP8 ? HB_POLY_MASK_FP8 : HB_POLY_MASK;
+                            if ((i & PM) == PM) {
+                                p = ex2_poly2<FP8 ? HB_POLY_DEG_FP8 : HB_POLY_DEG>(x);  // a fixed share of the pairs runs on the FMA pipes
                             } else {
                                 p.x = ex2(x.x);
                                 p.y = ex2(x.y);
