@@ -157,8 +157,9 @@ int hilberta_plan_export(const hilberta_plan_t *plan, int what, void *host_buf, 
  *   head_dim       bf16: 128 or 64.  fp32: 32, 64 or 128.  e4m3: 128.  Others: ERR_UNSUPPORTED.
  *   dtype          HILBERTA_BF16 (tensor-core kernel), HILBERTA_FP32 (plain FMA kernel) or
  *                  HILBERTA_FP8_E4M3 (tensor-core kernel, 8-bit operands, bf16 output; forward,
- *                  forward_lse, forward_unpermute and forward_fused only -- hilberta_backward*
- *                  and hilberta_forward_host return ERR_UNSUPPORTED).
+ *                  forward only: forward, forward_lse, forward_unpermute, forward_fused and
+ *                  forward_host (8-bit q, k, v in, bf16 out) -- hilberta_backward* return
+ *                  ERR_UNSUPPORTED).
  *   stride_b, stride_h, stride_s
  *                  element strides of q, k, v and out (all four share them) for
  *                  the batch, head and token axes; the head_dim axis is contiguous.
@@ -268,7 +269,8 @@ int hilberta_forward_unpermute(const void *q, const void *k, const void *v, void
 /* Entry gather of Sec. 3.4 (reordering is one row gather through the Hilbert table):
  *   dst[b, p, :] = src[b, phys2orig[p], :]   for b < batch, p < S.
  * src is in ORIGINAL order, dst in PHYSICAL order; both device pointers to
- * [batch, S, row_elems] contiguous arrays of `dtype`; rows must be a multiple of
+ * [batch, S, row_elems] contiguous arrays of `dtype` (any of the three element
+ * types; only the element size matters); rows must be a multiple of
  * 16 bytes and both pointers 16-byte aligned; src and dst must not overlap.
  * Asynchronous on `stream`. */
 int hilberta_permute(const void *src, void *dst, const hilberta_plan_t *plan, int batch,
@@ -289,7 +291,7 @@ int hilberta_unpermute(const void *src, void *dst, const hilberta_plan_t *plan, 
  *   out_original != 0 : `out` is written in ORIGINAL order (as
  *                       hilberta_forward_unpermute does).
  * With both flags zero this is hilberta_forward.  Same shapes, strides, alignment,
- * stream and error rules as hilberta_forward; bf16 and fp32 bindings. */
+ * stream and error rules as hilberta_forward; bf16, e4m3 and fp32 bindings. */
 int hilberta_forward_fused(const void *q, const void *k, const void *v, void *out,
                            const hilberta_plan_t *plan, int in_original, int out_original, void *stream);
 

@@ -826,12 +826,13 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     const bool fp8 = p->dtype == HILBERTA_FP8_E4M3;
     if (chunk >= 0 && p->chunk_heads < p->heads) {
         // a slice of heads: same strides, shifted base pointers, the slice's own schedule
-        if (lse || fp8) return HILBERTA_ERR_INVALID;
+        if (lse) return HILBERTA_ERR_INVALID;
         heads = p->chunk_heads;
-        const long long off = (long long)chunk * heads * p->stride_h;
-        q = (const __nv_bfloat16 *)q + off;
-        k = (const __nv_bfloat16 *)k + off;
-        v = (const __nv_bfloat16 *)v + off;
+        const long long off = (long long)chunk * heads * p->stride_h;   // elements
+        const long long esz_in = fp8 ? 1 : 2;
+        q = (const char *)q + off * esz_in;
+        k = (const char *)k + off * esz_in;
+        v = (const char *)v + off * esz_in;
         out = (__nv_bfloat16 *)out + off;
         units = p->d_units_chunk;
         cta_begin = p->d_cta_begin_chunk;

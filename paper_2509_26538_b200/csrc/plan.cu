@@ -687,9 +687,10 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
     int dev = -1;
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;
-    if (p->dtype == HILBERTA_FP8_E4M3) return HILBERTA_ERR_UNSUPPORTED;  // input and output element sizes differ
-    const size_t esz = p->dtype == HILBERTA_BF16 ? 2 : 4;
-    const size_t bytes = (size_t)p->batch * p->heads * p->S * p->head_dim * esz;
+    // element sizes of q, k, v and of out (e4m3 bindings: 8-bit inputs, bf16 output)
+    const size_t esz = p->dtype == HILBERTA_BF16 ? 2 : p->dtype == HILBERTA_FP8_E4M3 ? 1 : 4;
+    const size_t esz_out = p->dtype == HILBERTA_FP8_E4M3 ? 2 : esz;
+    const size_t bytes = (size_t)p->batch * p->heads * p->S * p->head_dim * esz_out;   // the larger of the two
     const size_t slot = (bytes + 255) & ~(size_t)255;
     if (p->ws_bytes < 4 * slot) {
         cudaFree(p->ws);
@@ -699,7 +700,7 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
         p->ws_bytes = 4 * slot;
     }
     // fp32 bindings have no slice schedule to build: chunk_heads is only set by the bf16 path
-    const int hc = (p->dtype == HILBERTA_BF16 && p->chunk_heads > 0) ? p->chunk_heads : p->heads;
+    const int hc = (p->dtype != HILBERTA_FP32 && p->chunk_heads > 0) ? p->chunk_heads : p->heads;
     const int n_chunks = p->heads / hc;
     if (!p->s_in) HB_CUDA(cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking));
     if (!p->s_out) HB_CUDA(cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking));
@@ -718,6 +719,7 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
     // a slice of hc heads of every batch item: `batch` rows of row_bytes, one tensor of heads apart
     const size_t row_bytes = (size_t)hc * p->S * p->head_dim * esz;
     const size_t pitch = (size_t)p->heads * p->S * p->head_dim * esz;
+    const size_t row_bytes_out = row_bytes / esz * esz_out, pitch_out = pitch / esz * esz_out;
     // work already queued on the caller's stream comes first
     HB_CUDA(cudaEventRecord(p->ev_in[n_chunks], st));
     HB_CUDA(cudaStreamWaitEvent(p->s_in, p->ev_in[n_chunks], 0));
@@ -733,7 +735,8 @@ extern "C" int hilberta_forward_host(const void *q, const void *k, const void *v
         if (rc != HILBERTA_OK) return rc;
         HB_CUDA(cudaEventRecord(p->ev_done[c], st));
         HB_CUDA(cudaStreamWaitEvent(p->s_out, p->ev_done[c], 0));
-        HB_CUDA(cudaMemcpy2DAsync((char *)out + off, pitch, out_dev + off, pitch, row_bytes, p->batch,
+        const size_t off_out = (size_t)c * row_bytes_out;
+        HB_CUDA(cudaMemcpy2DAsync((char *)out + off_out, pitch_out, out_dev + off_out, pitch_out, row_bytes_out, p->batch,
                                   cudaMemcpyDeviceToHost, p->s_out));
     }
     HB_CUDA(cudaStreamSynchronize(p->s_out));
