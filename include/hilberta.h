@@ -299,7 +299,7 @@ int hilberta_forward_fused(const void *q, const void *k, const void *v, void *ou
  * memory: copies q, k, v (HOST pointers, ORIGINAL order, dense
  * [batch, heads, S, head_dim]) to the device, runs hilberta_forward_fused with both
  * gathers fused in and copies the result to `out` (HOST pointer, ORIGINAL order).
- * The heads are processed in up to four slices whose copies (two internal copy
+ * The heads are processed in up to eight slices whose copies (two internal copy
  * streams, one per direction) and launches (`stream`) overlap.
  * Uses a device workspace that the first call on a plan allocates (and
  * hilberta_plan_destroy frees).  Requires a dense binding (strides 0).  The

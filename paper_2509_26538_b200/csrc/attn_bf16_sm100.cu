@@ -70,6 +70,9 @@ constexpr float P_SHIFT_FP8 = 4.0f;
 #ifndef HB_POLY_DEG
 #define HB_POLY_DEG 3
 #endif
+#ifndef HB_HOST_SLICES
+#define HB_HOST_SLICES 8   // hilberta_forward_host pipelines its copies and launches over about this many slices of heads
+#endif
 #ifndef HB_SPLIT_P
 #define HB_SPLIT_P 1     // hand P to the MMA issuer in two halves
 #endif
@@ -781,9 +784,9 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
     HB_CUDA(cudaMemcpy(p->d_work, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
     int rc = upload_schedule(items, cost, p->batch * p->heads, p->sm_count, &p->d_units, &p->d_cta_begin, &p->n_cta);
     if (rc != HILBERTA_OK) return rc;
-    // slice of heads for the pipelined host-buffer path: the divisor of `heads` nearest to a quarter
+    // slice of heads for the pipelined host-buffer path: the largest divisor of `heads` not above heads / HB_HOST_SLICES (rounded up)
     p->chunk_heads = p->heads;
-    for (int d = (p->heads + 3) / 4; d >= 1; --d)
+    for (int d = (p->heads + HB_HOST_SLICES - 1) / HB_HOST_SLICES; d >= 1; --d)
         if (p->heads % d == 0) {
             p->chunk_heads = d;
             break;
