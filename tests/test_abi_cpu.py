@@ -29,6 +29,19 @@ def test_every_declared_symbol_is_exported(lib):
         assert hasattr(lib, n), n
 
 
+def test_binding_constants_match_the_header():
+    """Element types, error codes and export selectors are spelled twice (header, binding): same values."""
+    text = open(os.path.join(ROOT, "include", "hilberta.h")).read()
+    defs = {m.group(1): int(m.group(2).strip("()"), 0)
+            for m in re.finditer(r"^#define\s+HILBERTA_([A-Z0-9_]+)\s+(\(?-?\d+\)?)\s", text, flags=re.M)}
+    for name in ("BF16", "FP32", "FP8_E4M3", "ERR_INVALID", "ERR_UNSUPPORTED", "ERR_ARCH", "ERR_CUDA", "ERR_NOMEM",
+                 "ERR_BUFFER", "ERR_UNBOUND", "ERR_TIMEOUT", "EXPORT_HIL_D2T", "EXPORT_HIL_T2D", "EXPORT_PHYS2ORIG",
+                 "EXPORT_ORIG2PHYS", "EXPORT_SHARED_RUNS", "EXPORT_WINDOWS", "EXPORT_NNZ", "EXPORT_INFO"):
+        assert name in defs, name
+        assert getattr(binding, name) == defs[name], name
+    assert len({defs["BF16"], defs["FP32"], defs["FP8_E4M3"]}) == 3
+
+
 def test_version_and_status_strings(lib):
     assert lib.hilberta_version() == 100
     seen = set()
