@@ -15,13 +15,16 @@
 //   warps 4-7  softmax + epilogue for query tile 1
 //   warp  8    TMA producer (one elected lane)
 //   warp  9    MMA issuer   (one elected lane)
-//   warps 10-11 idle; their registers go to the softmax warps (setmaxnreg)
+//   warps 10-11 idle (their registers go to the softmax warps, setmaxnreg); in the GATHER
+//               instantiations they are the loaders that fetch tile rows through the permutation
 // The two query tiles ping-pong: while one tile's softmax runs on the CUDA
 // cores, the tensor cores work on the other tile's P V and next Q K^T.
 // TMEM columns: S_t = Q_t K^T (fp32) at [128 t, 128 t + 128), overwritten in
 // place by P_t (bf16, first 64 columns); O_t accumulators at [256 + 128 t, +128).
 // The running maximum is only advanced when it grows by more than 2^8, so the
 // O accumulator is rescaled rarely; exponentials stay below 2^8.
+// FP8 instantiations take q, k, v as e4m3 bytes (128-byte rows, one slab per tile), round the
+// weights to e4m3 (four per TMEM column) and use kind::f8f6f4 MMAs; everything else is shared.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
