@@ -16,6 +16,10 @@
  *     kernels return ERR_INVALID if another device is current.
  *   - `stream` arguments are a cudaStream_t passed as void* (NULL = default
  *     stream).
+ *   - hilberta_forward, _forward_unpermute, _forward_fused, _forward_lse, _permute and
+ *     _unpermute only enqueue kernels on `stream`: no allocation, no synchronisation,
+ *     tensor maps passed to the kernels by value.  A sequence of them can be captured
+ *     into a CUDA graph and replayed.
  *   - ORIGINAL token order:  [ text 0..n_text ) ++ [ image tokens row-major,
  *     token n_text + r*W + c ].
  *   - PHYSICAL token order (the layout of Appendix A):
