@@ -102,6 +102,8 @@ def test_degenerate_and_maximum():
     _check(2, 4, 1, 2, 0)          # every image token shared
     _check(16, 256, 5, 16, 4)      # shared region = whole grid, one tile
     _check(512, 4096, 2048, 64, 512)  # 262144 image tokens
+    _check(1024, 4096, 2048, 64, 512)  # the largest grid the library accepts: 1048576 image tokens
+    _check(1000, 16384, 777, 10, 5, W=1024)  # the largest padded side with a ragged real grid
 
 
 def test_export_buffer_protocol():
