@@ -201,3 +201,30 @@ def test_general_shapes_elementwise(H, W, tile, o, hs, nt):
     ig, grp = orc.token_classes(H, W, tile, o, hs, nt)
     ref = attn_c.attention_rows(q.float().numpy(), k.float().numpy(), v.float().numpy(), ig, grp)
     check(got, ref)
+
+
+def test_largest_grid_one_head_sampled_rows():
+    """1024 x 1024 image tokens + 512 text (S = 1 049 088, the largest grid the plan accepts), one head:
+    64-bit row offsets, 8196 key blocks per prefix row, thousands of work units.  Sampled rows by the
+    oracle; the fused-gather launch must write the same bytes."""
+    H = W = 1024
+    tile, o, hs, nt = 4096, 2048, 64, 512
+    S = nt + H * W
+    g = torch.Generator().manual_seed(99)
+    q, k, v = (torch.randn((1, 1, S, 128), generator=g).bfloat16() for _ in range(3))
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    try:
+        got = run_gpu(plan, q, k, v, twice=False)
+        qd, kd, vd = (t.cuda() for t in (q, k, v))
+        of = torch.full_like(qd, float("nan"))
+        plan.bind_like(qd)
+        plan.forward_fused(qd, kd, vd, of, in_original=True, out_original=True)
+        assert plan.status() == 0
+        assert torch.equal(of.cpu().view(torch.int16), got.view(torch.int16))
+    finally:
+        plan.destroy()
+    rows = [0, nt - 1, nt, nt + 1, S - 1, S // 2, nt + 1024 * 512 + 512, nt + 1024 * 480 + 490, 777777, 123456]
+    ig, grp = orc.token_classes(H, W, tile, o, hs, nt)
+    ref = attn_c.attention_rows(q.float().numpy(), k.float().numpy(), v.float().numpy(), ig, grp, rows=rows)
+    check(got[:, :, rows], ref)
+    assert torch.isfinite(got.float()).all()

@@ -265,3 +265,39 @@ def test_backward_identities_at_full_size(name):
         assert ((a - b).abs() <= 2.0 ** -6 * size).all()
     finally:
         plan.destroy()
+
+
+def test_backward_largest_grid_one_head_identities():
+    """1024 x 1024 image tokens + 512 text (S = 1 049 088, the largest grid the plan accepts), one
+    head (64-bit offsets, 8196-block units).  At this size the oracle's backward pass, which visits
+    every (query, key) pair of the sequence, takes minutes, so the gradients are checked through the
+    identities that hold at any size (see test_backward_identities_at_full_size); parity against the
+    oracle at large sizes is test_backward_flux2048_sampled."""
+    H = W = 1024
+    tile, o, hs, nt = 4096, 2048, 64, 512
+    S = nt + H * W
+    g = torch.Generator(device="cuda").manual_seed(1234)
+    qp, kp, vp, dop = (torch.randn((1, 1, S, 128), generator=g, device="cuda").to(torch.bfloat16) for _ in range(4))
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    try:
+        out = torch.empty_like(qp)
+        lse = torch.empty((1, 1, S), device="cuda", dtype=torch.float32)
+        plan.bind_like(qp)
+        plan.forward_lse(qp, kp, vp, out, lse)
+        dq, dk, dv = (torch.full_like(qp, float("nan")) for _ in range(3))
+        plan.backward(dop, qp, kp, vp, out, lse, dq, dk, dv)
+        assert plan.status() == 0
+        for t in (dq, dk, dv):
+            assert torch.isfinite(t.float()).all()
+        dkf, dvf = dk.double(), dv.double()
+        tol_k = (S ** 0.5) * 2.0 ** -8 * dkf.pow(2).mean().sqrt()
+        assert dkf.sum(dim=2).abs().max() <= 4 * tol_k
+        want = dop.double().sum(dim=2)
+        tol_v = (S ** 0.5) * 2.0 ** -8 * max(dvf.pow(2).mean().sqrt(), dop.double().pow(2).mean().sqrt())
+        assert (dvf.sum(dim=2) - want).abs().max() <= 4 * tol_v
+        a = (qp.double() * dq.double()).sum(dim=(2, 3))
+        b = (kp.double() * dkf).sum(dim=(2, 3))
+        size = (qp.double() * dq.double()).abs().sum(dim=(2, 3))
+        assert ((a - b).abs() <= 2.0 ** -6 * size).all()
+    finally:
+        plan.destroy()
