@@ -45,7 +45,7 @@ def _draw(rng):
     return dict(kind=kind, H=H, W=W, F=F, tile=tile, groups=0, o=o, hs=hs, fs=fs, nt=nt)
 
 
-@pytest.mark.parametrize("seed", list(range(24)))
+@pytest.mark.parametrize("seed", list(range(48)) + [134, 188])   # 39, 134, 188: few-key rows with |O| > 2
 def test_random_configuration(seed):
     rng = np.random.default_rng(4242 + seed)
     c = _draw(rng)
@@ -86,7 +86,12 @@ def test_random_configuration(seed):
         assert plan.status() == 0, c
         got = out.cpu().double().numpy()
         assert np.isfinite(got).all(), c
-        assert orc.max_abs_err(got, ref_o) <= 1e-2 and orc.rel_l2_err(got, ref_o) <= 5e-3, c
+        # max-abs 1e-2 is a bar for outputs of size <= 1 (averages over many keys).  Tiny tiles give
+        # rows of 2 ... 20 keys whose outputs reach |O| = 2 ... 4, where bf16 values are 2^-6 apart:
+        # rounding the exact result alone errs by up to 7.8e-3 there, and the bf16 weights add
+        # 2^-9 |v|.  The bar therefore grows with |O| above 1: |err| <= 1e-2 max(1, |O|).
+        assert (np.abs(got - ref_o) <= 1e-2 * np.maximum(1.0, np.abs(ref_o))).all(), c
+        assert orc.rel_l2_err(got, ref_o) <= 5e-3, c
         for t, r in zip(grads, ref_g):
             full = torch.empty((1, heads, S, 128), dtype=torch.float64)
             full[:, :, p2o] = t.cpu().double()
