@@ -101,3 +101,68 @@ def test_random_configuration(seed):
             assert orc.max_abs_err(full.numpy(), r) <= 1e-2 * max(1.0, np.abs(r).max()), c
     finally:
         plan.destroy()
+
+
+@pytest.mark.parametrize("seed", list(range(18)))
+def test_random_configuration_other_element_types(seed):
+    """The same random configurations through the other kernels: bf16 with head dim 64, fp32 with head
+    dim 32 / 64 / 128 (forward and backward each) and e4m3 operands (forward), entry and exit gathers
+    fused into the forward launch."""
+    rng = np.random.default_rng(777 + seed)
+    c = _draw(rng)
+    H, W, F, tile, groups, o, hs, fs, nt = (c[k] for k in ("H", "W", "F", "tile", "groups", "o", "hs", "fs", "nt"))
+    S = nt + F * H * W
+    if S > 1400:
+        pytest.skip("plan-only size")
+    mode = ("bf16_64", "fp32", "e4m3")[seed % 3]
+    D = 64 if mode == "bf16_64" else (int(rng.choice([32, 64, 128])) if mode == "fp32" else 128)
+    dt = {"bf16_64": torch.bfloat16, "fp32": torch.float32, "e4m3": torch.float8_e4m3fn}[mode]
+    if groups:
+        ref = orc.plan_arrays_compact(H, W, groups, o, hs, nt)
+        ig, grp = orc.token_classes_compact(H, W, groups, o, hs, nt)
+    else:
+        ref = orc.plan_arrays(H, W, tile, o, hs, nt, frames=F, shared_frames=fs)
+        ig, grp = orc.token_classes(H, W, tile, o, hs, nt, frames=F, shared_frames=fs)
+    plan = hb.Plan(H, W, tile, o, hs, nt, groups=groups, frames=F, shared_frames=fs)
+    try:
+        g = torch.Generator().manual_seed(seed)
+        heads = int(rng.integers(1, 3))
+        q, k, v, do = (torch.randn((1, heads, S, D), generator=g).to(dt) for _ in range(4))
+        f32 = lambda t: t.float().numpy()
+        ref_o = attn_c.attention_rows(f32(q), f32(k), f32(v), ig, grp)
+        qd, kd, vd = (t.cuda() for t in (q, k, v))
+        plan.bind_like(qd)
+        out = torch.full((1, heads, S, D), float("nan"), device="cuda",
+                         dtype=torch.bfloat16 if mode == "e4m3" else dt)
+        plan.forward_fused(qd, kd, vd, out, in_original=True, out_original=True)
+        assert plan.status() == 0, c
+        got = out.cpu().double().numpy()
+        assert np.isfinite(got).all(), c
+        err = np.abs(got - ref_o)
+        if mode == "fp32":
+            assert err.max() <= 1e-5 * max(1.0, np.abs(ref_o).max()), c
+        elif mode == "e4m3":
+            assert orc.rel_l2_err(got, ref_o) <= 4e-2, c          # three mantissa bits in the weights
+            return                                                 # forward only
+        else:
+            assert (err <= 1e-2 * np.maximum(1.0, np.abs(ref_o))).all() and orc.rel_l2_err(got, ref_o) <= 5e-3, c
+        p2o = torch.from_numpy(ref["phys2orig"].astype(np.int64))
+        qp, kp, vp, dop = (t[:, :, p2o].contiguous().cuda() for t in (q, k, v, do))
+        ref_g = attn_c.attention_backward(f32(q), f32(k), f32(v), f32(do), ig, grp)
+        outp = torch.empty_like(qp)
+        lse = torch.empty((1, heads, S), device="cuda", dtype=torch.float32)
+        plan.bind_like(qp)
+        plan.forward_lse(qp, kp, vp, outp, lse)
+        grads = [torch.full_like(qp, float("nan")) for _ in range(3)]
+        plan.backward(dop, qp, kp, vp, outp, lse, *grads)
+        assert plan.status() == 0, c
+        tol_rel, tol_abs = (1e-5, 1e-5) if mode == "fp32" else (5e-3, 1e-2)
+        for t, r in zip(grads, ref_g):
+            full = torch.empty((1, heads, S, D), dtype=torch.float64)
+            full[:, :, p2o] = t.cpu().double()
+            assert np.isfinite(full.numpy()).all(), c
+            if np.abs(r).max() > 0:
+                assert orc.rel_l2_err(full.numpy(), r) <= tol_rel, c
+            assert orc.max_abs_err(full.numpy(), r) <= tol_abs * max(1.0, np.abs(r).max()), c
+    finally:
+        plan.destroy()
