@@ -154,6 +154,26 @@ __device__ __forceinline__ float2 ex2_poly2(float2 x) {
     return p;
 }
 
+// One lane of ex2_poly2 with scalar instructions: the same operations in the same order, hence the
+// same bits.
+template <int DEG = 3>
+__device__ __forceinline__ float ex2_poly1(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = __fadd_rn(x, 12582912.f);
+    const float n = __fadd_rn(t, -12582912.f);
+    const float f = __fadd_rn(x, -n);
+    float p;
+    if constexpr (DEG == 2) {
+        p = __fmaf_rn(f, 0.23842697f, 0.7034453f);
+        p = __fmaf_rn(p, f, 1.00044307f);
+    } else {
+        p = __fmaf_rn(f, 0.055088773f, 0.24260406f);
+        p = __fmaf_rn(p, f, 0.69327623f);
+        p = __fmaf_rn(p, f, 0.99992895f);
+    }
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
 // S_t = Q_t K^T for one 128-key block: HD / 16 MMAs of K = 16 (bf16) or HD / 32 of K = 32 (e4m3);
 // either way an MMA consumes 32 bytes of every row.
 template <int HD, bool FP8>
@@ -530,17 +550,27 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         for (int i = 0; i < BN; ++i)
                             if (i >= valid) s[i] = 0xff800000u;  // -inf
                     }
-                    // eight independent max chains, then a short tree
+                    // Eight independent max chains, then a short tree.  Chain c takes the pairs of scores
+                    // whose index is c modulo 8; with one pair in four on the polynomial (pairs 3 modulo
+                    // 4) chains 3 and 7 see exactly the scores whose exponentials the FMA pipes will
+                    // compute, the other six those of the MUFU unit -- the first eight scores seed the
+                    // chains accordingly (scores 6, 7 are pair 3; score 3 is pair 1).  So the block
+                    // maximum comes with the path its weight will take, at no cost.
+                    constexpr int PM = FP8 ? HB_POLY_MASK_FP8 : HB_POLY_MASK;
+                    static_assert(PM == 3 || PM == 0xff, "the chain seeding below assumes pairs 3 mod 4 (or none) on the polynomial");
                     float mxa[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) mxa[i] = __uint_as_float(s[i]);
+                    for (int i = 0; i < 8; ++i) mxa[i] = __uint_as_float(s[i == 3 ? 6 : (i == 6 ? 3 : i)]);
 #pragma unroll
                     for (int i = 8; i < BN; i += 2) {
                         const int c = (i >> 1) & 7;
                         mxa[c] = max3(mxa[c], __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
                     }
-                    float mx = max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7]));
-                    mx *= scale_log2;
+                    const float mx_fma = fmaxf(mxa[3], mxa[7]);
+                    const float mx_mufu = fmaxf(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[4], mxa[5], mxa[6]));
+                    const float mx_raw = fmaxf(mx_fma, mx_mufu);            // the block's largest score, unscaled
+                    const bool top_on_fma = PM == 3 && mx_fma > mx_mufu;    // ... and who computes its weight
+                    float mx = mx_raw * scale_log2;
                     if (first) {
                         m_ref = mx;
                         first = false;
@@ -567,16 +597,19 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     const float nm = FP8 ? P_SHIFT_FP8 - m_ref : -m_ref;
                     const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(nm, nm);
                     float2 sum[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-                    // The row sum is taken over the fp32 weights; the P V MMA sees them rounded
-                    // to bf16.  For the block's largest weight -- the one that dominates a
-                    // near-one-hot row -- the rounding error is added to the sum, so numerator
-                    // and denominator round together where it matters.
-                    if constexpr (FP8) {
-                        const float pm = ex2(mx + nm);
-                        l_fix += round_e4m3(pm) - pm;
-                    } else {
-                        const float pm = ex2(mx - m_ref);
-                        l += __uint_as_float(pack_bf16(0.f, pm) & 0xffff0000u) - pm;
+                    // The row sum is taken over the fp32 weights; the P V MMA sees them rounded.  For
+                    // the block's largest weight -- the one that dominates a near-one-hot row -- the
+                    // rounding error is added to the sum, so numerator and denominator round together
+                    // where it matters.  The weight is recomputed here exactly as the loop below will
+                    // compute it (same fused multiply-add, same exponential): the MUFU unit and the
+                    // polynomial agree to 8e-5 only, and a weight next to a rounding tie that rounded
+                    // one way here and the other way there would double the error instead of cancelling it.
+                    {
+                        const float xm = fmaf(mx_raw, scale_log2, nm);
+                        const float pm_fma = ex2_poly1<FP8 ? HB_POLY_DEG_FP8 : HB_POLY_DEG>(xm);
+                        const float pm = top_on_fma ? pm_fma : ex2(xm);
+                        if constexpr (FP8) l_fix += round_e4m3(pm) - pm;
+                        else l += __uint_as_float(pack_bf16(0.f, pm) & 0xffff0000u) - pm;
                     }
 #pragma unroll
                     for (int c = 0; c < BN / 32; ++c) {
@@ -588,7 +621,6 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                                                     __uint_as_float(s[c * 32 + 2 * i + 1])),
                                                         sc2, nm2);
                             float2 p;
-                            constexpr int PM = FP8 ? HB_POLY_MASK_FP8 : HB_POLY_MASK;
                             if ((i & PM) == PM) {
                                 p = ex2_poly2<FP8 ? HB_POLY_DEG_FP8 : HB_POLY_DEG>(x);  // a fixed share of the pairs runs on the FMA pipes
                             } else {
