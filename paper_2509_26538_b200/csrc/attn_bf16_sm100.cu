@@ -528,7 +528,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const int bh = unit.bh;
             const int b = bh / prm.heads, h = bh % prm.heads;
             float m_ref = 0.f, l = 0.f;
-            float l_fix = 0.f;   // e4m3 only: rounding error of every block's largest weight (kept out of lse)
+            float l_fix = 0.f;   // rounding errors of the blocks' largest weights: part of the output's normaliser, not of lse
             bool first = true;
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                 const int nb = item_blocks(wi, seg);
@@ -583,7 +583,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         const float alpha = ex2(m_ref - m_new);
                         m_ref = m_new;
                         l *= alpha;
-                        if constexpr (FP8) l_fix *= alpha;
+                        l_fix *= alpha;
 #pragma unroll
                         for (int c = 0; c < HD / 32; ++c) {
                             uint32_t o[32];
@@ -609,7 +609,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         const float pm_fma = ex2_poly1<FP8 ? HB_POLY_DEG_FP8 : HB_POLY_DEG>(xm);
                         const float pm = top_on_fma ? pm_fma : ex2(xm);
                         if constexpr (FP8) l_fix += round_e4m3(pm) - pm;
-                        else l += __uint_as_float(pack_bf16(0.f, pm) & 0xffff0000u) - pm;
+                        else l_fix += __uint_as_float(pack_bf16(0.f, pm) & 0xffff0000u) - pm;
                     }
 #pragma unroll
                     for (int c = 0; c < BN / 32; ++c) {
@@ -664,7 +664,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             ok = wait_or_abort(bar(PV_DONE + t), (cPV - 1) & 1, &abort_flag, prm.status, 0x305 + t);
             if (!ok) break;
             tc_fence_after();
-            const float inv = 1.f / (FP8 ? l + l_fix : l);
+            const float inv = 1.f / (l + l_fix);
             const int row = t * BM + r;
             // each thread stores its own row, so writing it at its ORIGINAL position instead
             // of the physical one (the exit gather of Sec. 3.4 fused in) costs one index read
