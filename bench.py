@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 NOMINAL_BF16_TFLOPS = 2250.0
 L2_BYTES = 126 * 2**20   # B200 L2
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one forward launch, from the
-# ncu capture summarised in profiles/attn_bf16_kernel_flux2048.md (555.1 MB read + 92.4 MB written).
+# dram__bytes_read.sum + dram__bytes_write.sum of one forward launch (one ncu capture of the
+# single-CTA bf16 kernel at this workload: 555.1 MB read + 92.4 MB written).
 FORWARD_DRAM_TRAFFIC_BYTES = {"flux2048": 647.5e6}
 
 
@@ -50,10 +50,10 @@ class ClockSampler(threading.Thread):
     """Polls SM clock and throttle reasons through NVML (read-only) while the
     timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
-        self.samples, self.reasons = [], set()
+        self.samples, self.stamps, self.reasons = [], [], set()
         self.max_mhz = None
         self._stop_evt = threading.Event()
         self.ok = False
@@ -81,6 +81,7 @@ class ClockSampler(threading.Thread):
         while not self._stop_evt.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.stamps.append(time.perf_counter())
                 try:
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
@@ -92,11 +93,19 @@ class ClockSampler(threading.Thread):
                 pass
             time.sleep(self.period)
 
-    def stop(self):
+    def stop(self, window=None):
+        """window = (t0, t1) in time.perf_counter() seconds: also report the samples taken inside it."""
         self._stop_evt.set()
         self.join(timeout=2)
-        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        out = {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+               "sm_min_mhz": min(self.samples) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
+               "period_ms": 1e3 * self.period}
+        if window:
+            inside = [m for m, t in zip(self.samples, self.stamps) if window[0] <= t <= window[1]]
+            out["samples_in_timed_region"] = len(inside)
+            out["sm_mhz_in_timed_region"] = statistics.median(inside) if inside else None
+        return out
 
 
 def oracle_sample(wl, seconds_target: float, heads: int = 2):
@@ -209,10 +218,25 @@ def main():
     ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass row")
     ap.add_argument("--no-fp8", action="store_true", help="skip the e4m3-operand forward row")
     ap.add_argument("--schedule", action="store_true",
-                    help="also time the 57-layer per-step schedule (one permute, 57 forwards with the "
-                         "per-layer offsets, one unpermute) on the chosen workload's shape")
+                    help="time the 57-layer per-step schedule (one permute, 57 forwards with the per-layer "
+                         "offsets, one unpermute) on the chosen workload's shape instead of the 1024^2 one")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the rows for the other workload sizes (1024^2 tile sweep, 4096^2) and the 57-layer schedule")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the 2-second back-to-back row")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: 'replicas' = one independent batch per GPU (weak scaling); 'heads' = one batch whose "
+                         "(batch, head) units are split across the GPUs (strong scaling); no collective either way")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: become N ranks (one per GPU) of a single-node job
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                   f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+                                   "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:])
 
     from paper_2509_26538_b200.inputs import WORKLOADS, make_qkv
     wl = WORKLOADS[args.workload]
@@ -251,8 +275,20 @@ def main():
         dist.barrier()
 
     peaks = load_peaks()
-    # ---- inputs: seeded, one independent batch per rank, resident in HBM
-    q, k, v = make_qkv(wl.with_(seed=wl.seed + 100 * rank))
+    # ---- inputs: seeded, resident in HBM.  replicas: one independent batch per rank; heads: every rank
+    # takes its contiguous slice of the (batch, head) units of ONE batch (no data is exchanged)
+    shard_heads = distributed and args.shard == "heads"
+    if shard_heads:
+        from paper_2509_26538_b200.sharding import unit_slice
+        if wl.batch != 1:
+            raise SystemExit("--shard heads expects batch 1")
+        h0, h1 = unit_slice(wl.heads, world, rank)
+        q, k, v = (t[:, h0:h1].contiguous() for t in make_qkv(wl))
+        full_heads = wl.heads
+        wl = wl.with_(heads=h1 - h0)
+    else:
+        q, k, v = make_qkv(wl.with_(seed=wl.seed + 100 * rank))
+        full_heads = wl.heads * (world if distributed else 1)
     qd, kd, vd = (t.cuda() for t in (q, k, v))
     qp, kp, vp, op, od = (torch.empty_like(qd) for _ in range(5))
     # Workloads whose tensors fit in L2 (126 MB) rotate through several copies of the step's

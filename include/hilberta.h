@@ -79,6 +79,7 @@ extern "C" {
 #define HILBERTA_EXPORT_WINDOWS 5     /* int32[T][5] per slid tile: lo, seg0_start, seg0_len, seg1_start, seg1_len */
 #define HILBERTA_EXPORT_NNZ 6         /* uint64[1]   number of (query, key) pairs the mask keeps */
 #define HILBERTA_EXPORT_INFO 7        /* int32[11]   H, W, tile, offset mod NP, shared_region, n_text, n_shared, T, padded side n, frames, shared_frames */
+#define HILBERTA_EXPORT_LAUNCH_CLOCK 8 /* int32[2]  SM cycles and nanoseconds that the first CTA of the plan's latest tensor-core forward launch was resident: cycles / ns = the SM clock (GHz) that launch ran at; synchronises the device */
 
 typedef struct hilberta_plan_s hilberta_plan_t;
 

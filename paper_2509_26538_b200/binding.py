@@ -19,7 +19,7 @@ ERR_INVALID, ERR_UNSUPPORTED, ERR_ARCH, ERR_CUDA, ERR_NOMEM, ERR_BUFFER, ERR_UNB
     -1, -2, -3, -4, -5, -6, -7, -8)
 BF16, FP32, FP8_E4M3 = 0, 1, 2
 (EXPORT_HIL_D2T, EXPORT_HIL_T2D, EXPORT_PHYS2ORIG, EXPORT_ORIG2PHYS, EXPORT_SHARED_RUNS, EXPORT_WINDOWS,
- EXPORT_NNZ, EXPORT_INFO) = range(8)
+ EXPORT_NNZ, EXPORT_INFO, EXPORT_LAUNCH_CLOCK) = range(9)
 
 # every symbol include/hilberta.h declares
 SYMBOLS = (
@@ -130,7 +130,7 @@ _EXPORT_NP = {
     EXPORT_HIL_D2T: (np.int32, None), EXPORT_HIL_T2D: (np.int32, None),
     EXPORT_PHYS2ORIG: (np.int32, None), EXPORT_ORIG2PHYS: (np.int32, None),
     EXPORT_SHARED_RUNS: (np.int32, 2), EXPORT_WINDOWS: (np.int32, 5),
-    EXPORT_NNZ: (np.uint64, None), EXPORT_INFO: (np.int32, None),
+    EXPORT_NNZ: (np.uint64, None), EXPORT_INFO: (np.int32, None), EXPORT_LAUNCH_CLOCK: (np.int32, None),
 }
 
 

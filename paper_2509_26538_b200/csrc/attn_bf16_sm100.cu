@@ -29,12 +29,14 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <functional>
 #include <mutex>
 #include <queue>
 #include <type_traits>
 #include <utility>
 
+#include "attn_softmax_math.cuh"
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -61,17 +63,11 @@ constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 // the smallest nonzero one, 2^-9, is 2^-13 of the reference maximum.
 constexpr float RESCALE_THRESHOLD_FP8 = 4.0f;
 constexpr float P_SHIFT_FP8 = 4.0f;
-#ifndef HB_POLY_MASK
-#define HB_POLY_MASK 3   // pair i of every 16 runs its two exponentials on the FMA pipes when (i & MASK) == MASK (3: one pair in four); 0xff = never
-#endif
 #ifndef HB_POLY_MASK_FP8
 #define HB_POLY_MASK_FP8 HB_POLY_MASK
 #endif
 #ifndef HB_POLY_DEG_FP8
 #define HB_POLY_DEG_FP8 2
-#endif
-#ifndef HB_POLY_DEG
-#define HB_POLY_DEG 3
 #endif
 #ifndef HB_HOST_SLICES
 #define HB_HOST_SLICES 8   // hilberta_forward_host pipelines its copies and launches over about this many slices of heads
@@ -120,58 +116,6 @@ struct KernelParams<true> : Params {
 
 __device__ __forceinline__ int item_blocks(const WorkItem &it, int seg) {
     return (it.seg_len[seg] + BN - 1) / BN;
-}
-
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float y;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
-    return y;
-}
-
-// 2^x for a pair of values on the FMA pipes (no MUFU), with packed fp32x2 instructions:
-// x = n + f with n = round(x) (adding 1.5 * 2^23 leaves the integer in the low mantissa
-// bits), f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.8e-5, far below bf16
-// rounding), 2^n by an exponent add.  Used for a fixed share of the exponentials so that
-// the MUFU unit and the FMA pipes split the work.  x is clamped at -126 (result ~0).
-template <int DEG = 3>
-__device__ __forceinline__ float2 ex2_poly2(float2 x) {
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
-    const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-    float2 p;
-    if constexpr (DEG == 2) {
-        p = __ffma2_rn(f, make_float2(0.23842697f, 0.23842697f), make_float2(0.7034453f, 0.7034453f));
-        p = __ffma2_rn(p, f, make_float2(1.00044307f, 1.00044307f));
-    } else {
-        p = __ffma2_rn(f, make_float2(0.055088773f, 0.055088773f), make_float2(0.24260406f, 0.24260406f));
-        p = __ffma2_rn(p, f, make_float2(0.69327623f, 0.69327623f));
-        p = __ffma2_rn(p, f, make_float2(0.99992895f, 0.99992895f));
-    }
-    p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
-    p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
-    return p;
-}
-
-// One lane of ex2_poly2 with scalar instructions: the same operations in the same order, hence the
-// same bits.
-template <int DEG = 3>
-__device__ __forceinline__ float ex2_poly1(float x) {
-    x = fmaxf(x, -126.f);
-    const float t = __fadd_rn(x, 12582912.f);
-    const float n = __fadd_rn(t, -12582912.f);
-    const float f = __fadd_rn(x, -n);
-    float p;
-    if constexpr (DEG == 2) {
-        p = __fmaf_rn(f, 0.23842697f, 0.7034453f);
-        p = __fmaf_rn(p, f, 1.00044307f);
-    } else {
-        p = __fmaf_rn(f, 0.055088773f, 0.24260406f);
-        p = __fmaf_rn(p, f, 0.69327623f);
-        p = __fmaf_rn(p, f, 0.99992895f);
-    }
-    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
 }
 
 // S_t = Q_t K^T for one 128-key block: HD / 16 MMAs of K = 16 (bf16) or HD / 32 of K = 32 (e4m3);
@@ -236,6 +180,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __shared__ uint64_t bars[NUM_BARS];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ long long stamp[2];
     static_assert(!FP8 || HD == 128, "e4m3 operands: head dim 128 only");
     constexpr int TILE_BYTES = tile_bytes(HD, FP8);
     constexpr int NSLAB = TILE_BYTES / SLAB_BYTES;
@@ -269,6 +214,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     const int u_begin = prm.cta_begin[blockIdx.x], u_end = prm.cta_begin[blockIdx.x + 1];
+    if (blockIdx.x == 0 && tid == 0) {
+        // start stamps of the launch's first CTA (kept in shared memory: no register lives across the kernel)
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        stamp[0] = clock64();
+        stamp[1] = (long long)ns;
+    }
 
     // Registers move from the data-movement warpgroup to the two softmax warpgroups.  The split
     // is tuned: spills in the MMA issuer (fewer than 88) or in the softmax warps (fewer than
@@ -716,6 +668,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
+    if (blockIdx.x == 0 && tid == 0) {
+        // elapsed SM cycles and nanoseconds of this CTA: the launch's effective SM clock
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        prm.status[32] = (int)(clock64() - stamp[0]);
+        prm.status[33] = (int)((long long)ns - stamp[1]);
+    }
     if (warp == 8) {
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
@@ -831,33 +790,38 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
                              &p->n_cta_chunk);
         if (rc != HILBERTA_OK) return rc;
     }
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            smem_bytes(128));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            smem_bytes(64));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            smem_bytes(64));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<false, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            smem_bytes(128, true));
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_bf16_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            smem_bytes(128, true));
-    });
-    HB_CUDA(attr_err);
-    return HILBERTA_OK;
+    {
+        // The shared-memory opt-in is an attribute of the kernel ON ONE DEVICE: set it once for every
+        // device a plan is bound on (a failure is reported, not remembered).
+        static std::mutex attr_mutex;
+        static bool attr_done[64] = {};
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if (p->device < 0 || p->device >= 64) return HILBERTA_ERR_INVALID;
+        if (!attr_done[p->device]) {
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<false, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128, true)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128, true)));
+            attr_done[p->device] = true;
+        }
+    }
+    return attn_bf16_pair_prepare(p);
 }
 
 int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
                      float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk) {
     if (p->n_work == 0) return HILBERTA_OK;
+    // bf16 with head dim 128 and inputs in physical order can also run on pairs of SMs
+    // (attn_bf16_pair_sm100.cu).  That kernel is correct but measures slower than this one, so it is
+    // opt-in: the environment variable HILBERTA_FORWARD_KERNEL=pair selects it (read once).
+    static const bool use_pair = [] {
+        const char *e = getenv("HILBERTA_FORWARD_KERNEL");
+        return e && e[0] == 'p';
+    }();
+    if (use_pair && !in_map && chunk < 0 && p->n_pair > 0)
+        return launch_attn_bf16_pair(p, q, k, v, out, lse, out_map, stream);
     int heads = p->heads, n_cta = p->n_cta;
     const WorkUnit *units = p->d_units;
     const int *cta_begin = p->d_cta_begin;

@@ -92,6 +92,12 @@ struct hilberta_plan_s {
     hilberta::WorkUnit *d_units_chunk;
     int *d_cta_begin_chunk;
     int n_cta_chunk;
+    // the pair kernel's work list and schedule (bf16, head dim 128): items of 256 rows, one per
+    // pair of SMs; n_pair == 0: the shape is served by the single-CTA kernel
+    hilberta::WorkItem *d_work_pair;
+    hilberta::WorkUnit *d_units_pair;
+    int *d_pair_begin;
+    int n_pair;
     cudaStream_t s_in, s_out;           // copy streams of hilberta_forward_host (created on first use)
     std::vector<cudaEvent_t> ev_in, ev_done;
     // backward pass: 128-row items over the same key lists, their schedule, and the
@@ -128,6 +134,10 @@ std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, 
 int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
                     WorkUnit **d_units, int **d_cta_begin, int *n_cta_out);
 int attn_bf16_prepare(hilberta_plan_t *p);
+// attn_bf16_pair_sm100.cu: the forward kernel on pairs of SMs (bf16, head dim 128, inputs in physical order)
+int attn_bf16_pair_prepare(hilberta_plan_t *p);
+int launch_attn_bf16_pair(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
+                          float *lse, const int *out_map, cudaStream_t stream);
 int attn_bwd_prepare(hilberta_plan_t *p);
 // dq, dk, dv (bf16, physical order, the bound strides) from dout, q, k, v, out and the forward's lse.
 int launch_attn_bwd(const hilberta_plan_t *p, const void *dout, const void *q, const void *k, const void *v,

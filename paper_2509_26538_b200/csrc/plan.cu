@@ -286,6 +286,9 @@ static void free_plan(hilberta_plan_t *p) {
     cudaFree(p->d_units);
     cudaFree(p->d_cta_begin);
     cudaFree(p->d_units_chunk);
+    cudaFree(p->d_work_pair);
+    cudaFree(p->d_units_pair);
+    cudaFree(p->d_pair_begin);
     cudaFree(p->d_cta_begin_chunk);
     for (cudaEvent_t e : p->ev_in) cudaEventDestroy(e);
     for (cudaEvent_t e : p->ev_done) cudaEventDestroy(e);
@@ -547,6 +550,11 @@ extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *ho
                    p->frames, p->shared_frames};
             need = sizeof(int) * tmp.size();
             hsrc = tmp.data();
+            break;
+        case HILBERTA_EXPORT_LAUNCH_CLOCK:
+            need = sizeof(int) * 2;
+            dsrc = p->d_status + 32;
+            if (host_buf) HB_CUDA(cudaDeviceSynchronize());
             break;
 #ifdef HB_TIMING
         case 100: need = sizeof(int) * 4096; dsrc = p->d_status; break;  // role cycle counters and event trace

@@ -36,7 +36,7 @@ def test_binding_constants_match_the_header():
             for m in re.finditer(r"^#define\s+HILBERTA_([A-Z0-9_]+)\s+(\(?-?\d+\)?)\s", text, flags=re.M)}
     for name in ("BF16", "FP32", "FP8_E4M3", "ERR_INVALID", "ERR_UNSUPPORTED", "ERR_ARCH", "ERR_CUDA", "ERR_NOMEM",
                  "ERR_BUFFER", "ERR_UNBOUND", "ERR_TIMEOUT", "EXPORT_HIL_D2T", "EXPORT_HIL_T2D", "EXPORT_PHYS2ORIG",
-                 "EXPORT_ORIG2PHYS", "EXPORT_SHARED_RUNS", "EXPORT_WINDOWS", "EXPORT_NNZ", "EXPORT_INFO"):
+                 "EXPORT_ORIG2PHYS", "EXPORT_SHARED_RUNS", "EXPORT_WINDOWS", "EXPORT_NNZ", "EXPORT_INFO", "EXPORT_LAUNCH_CLOCK"):
         assert name in defs, name
         assert getattr(binding, name) == defs[name], name
     assert len({defs["BF16"], defs["FP32"], defs["FP8_E4M3"]}) == 3
