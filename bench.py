@@ -28,6 +28,10 @@ if ROOT not in sys.path:
 
 NOMINAL_BF16_TFLOPS = 2250.0
 L2_BYTES = 126 * 2**20   # B200 L2
+# Idle time before a side row is timed: the GPU's clock follows a moving average of its power draw
+# (1 kW cap), so a row measured right after seconds of full load runs at 1.3-1.5 GHz instead of the
+# 1.6-1.9 GHz a short run sees.  Every row also reports the SM clock its last launch ran at.
+COOL_DOWN_S = 1.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one forward launch (one ncu capture of the
 # single-CTA bf16 kernel at this workload: 555.1 MB read + 92.4 MB written).
@@ -163,6 +167,9 @@ def run_reference(args, wl):
     """CPU oracle arm: rank 0 only; other ranks exit without work."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
+    if "TORCHELASTIC_RUN_ID" in os.environ and os.environ.get("OMP_NUM_THREADS") == "1":
+        # torch.distributed.run pins every rank to one OpenMP thread; this arm runs on rank 0 alone
+        del os.environ["OMP_NUM_THREADS"]
     total_budget = 150.0
     per_step = max(0.05, min(20.0, total_budget / (args.steps + args.warmup + 1)))
     vals, times = [], []
@@ -187,7 +194,7 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(wl, n_gpus):
+def workload_config(wl, n_gpus, shard="replicas"):
     return {"workload": f"{wl.name}: {wl.H}x{wl.W} image tokens + {wl.n_text} text, batch {wl.batch} per GPU, "
                         f"{wl.heads} heads x {wl.head_dim}, tile {wl.tile}, shared {wl.shared_region}x"
                         f"{wl.shared_region}, offset {wl.layer_offset}",
@@ -196,7 +203,126 @@ def workload_config(wl, n_gpus):
             "l2": ("inputs larger than L2 (Q+K+V+O = %d MB)" if 4 * wl.batch * wl.heads * wl.S * wl.head_dim * 2 > L2_BYTES
                    else "Q+K+V+O = %d MB fits in L2: the steps rotate through several copies of their buffers") %
                   (4 * wl.batch * wl.heads * wl.S * wl.head_dim * 2 // 2**20),
-            "parallelism": f"replicas x{n_gpus} (independent batches, no collective)"}
+            "parallelism": (f"replicas x{n_gpus} (independent batches, no collective)" if shard == "replicas" else
+                            f"one batch, its (batch, head) units split over {n_gpus} GPUs ({wl.heads} heads on this rank), no collective")}
+
+
+def device_qkv(torch, wl, seed_offset=0):
+    """Q, K, V ~ N(0,1) drawn on the device from the workload's seed (the timing-only rows of the other
+    workload sizes; the parity tests and the main workload use the CPU draw of inputs.make_qkv)."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(wl.seed + seed_offset)
+    shape = (wl.batch, wl.heads, wl.S, wl.head_dim)
+    return tuple(torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(3))
+
+
+def n_buffer_sets(wl, tensors_per_set=4):
+    """Workloads whose tensors fit in L2 rotate through several copies so that no call finds its inputs cached."""
+    set_bytes = tensors_per_set * wl.batch * wl.heads * wl.S * wl.head_dim * 2
+    return 1 if set_bytes >= 2 * L2_BYTES else min(8, -(-3 * L2_BYTES // set_bytes))
+
+
+def time_forward_config(hb, torch, wl, peaks, stream, n_calls=30):
+    """ms per forward call (CUDA events around each launch) of one workload configuration."""
+    n_sets = n_buffer_sets(wl)
+    sets = [device_qkv(torch, wl, 17 * i) for i in range(n_sets)]   # used as if already in physical order
+    out = torch.empty_like(sets[0][0])
+    t0 = time.perf_counter()
+    plan = hb.Plan(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
+    plan.bind_like(out)
+    torch.cuda.synchronize()
+    plan_ms = 1e3 * (time.perf_counter() - t0)
+    nnz = int(plan.export(hb.EXPORT_NNZ)[0])
+    flops = 4.0 * wl.head_dim * wl.heads * wl.batch * nnz
+    for i in range(4):
+        plan.forward(*sets[i % n_sets], out)
+    torch.cuda.synchronize()
+    time.sleep(COOL_DOWN_S)   # the rows before this one ran the GPU into its power cap
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_calls)]
+    for i, (a, b_) in enumerate(ev):
+        a.record(stream)
+        plan.forward(*sets[i % n_sets], out)
+        b_.record(stream)
+    torch.cuda.synchronize()
+    assert plan.status() == 0, "device-side wait timed out"
+    assert torch.isfinite(out.float()).all()
+    lc = plan.export(hb.EXPORT_LAUNCH_CLOCK)
+    ms = sorted(a.elapsed_time(b_) for a, b_ in ev)
+    med = ms[len(ms) // 2]
+    tf = flops / (med * 1e-3) / 1e12
+    plan.destroy()
+    del sets, out
+    torch.cuda.empty_cache()
+    return {"workload": "%s: %dx%d + %d text, %d heads x %d, tile %d, shared %d, offset %d" % (
+                wl.name, wl.H, wl.W, wl.n_text, wl.heads, wl.head_dim, wl.tile, wl.shared_region, wl.layer_offset),
+            "ms_per_call_median": med, "ms_per_call_min": ms[0], "useful_tflops": tf, "nnz": nnz,
+            "useful_gflop_per_call": flops / 1e9,
+            "frac_of_measured_burst_peak": tf / peaks["bf16_tflops"],
+            "frac_of_measured_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_peak": tf / NOMINAL_BF16_TFLOPS,
+            "effective_sm_mhz_last_launch": (1e3 * float(lc[0]) / float(lc[1])) if lc[1] > 0 else None,
+            "buffer_sets": n_sets, "calls": n_calls, "plan_build_ms": plan_ms,
+            "data": "synthetic, N(0,1) drawn on the device"}
+
+
+def run_schedule57(hb, torch, wl, stream, steps):
+    """The full per-step layer schedule (Sec. 3.4 with the per-layer offsets of Sec. 3.2): one entry
+    permute of Q, K, V, 57 attention layers whose offsets are (layer * tile / 4) mod HW, the last of
+    which writes its output in the original order."""
+    from paper_2509_26538_b200.inputs import SCHEDULE_LAYERS, schedule_offset
+    n_sets = max(4, n_buffer_sets(wl, 3))
+    qd, kd, vd = device_qkv(torch, wl)                       # original order
+    qp, kp, vp, op, od = (torch.empty_like(qd) for _ in range(5))
+    layer_sets = [device_qkv(torch, wl, 31 * (i + 1)) for i in range(n_sets)]   # the layers' own activations
+    offs = [schedule_offset(layer, wl.tile, wl.HW) for layer in range(SCHEDULE_LAYERS)]
+    # only offset mod tile changes the mask: the 57 layers share a few plans
+    offs = [o % wl.tile for o in offs]
+    plans = {}
+    for o in sorted(set(offs)):
+        plans[o] = hb.Plan(wl.H, wl.W, wl.tile, o, wl.shared_region, wl.n_text)
+        plans[o].bind_like(qp)
+    any_plan = plans[offs[0]]
+    sched_flops = sum(4.0 * wl.head_dim * wl.heads * wl.batch * int(plans[o].export(hb.EXPORT_NNZ)[0]) for o in offs)
+
+    def sched_step():
+        # the physical layout does not depend on the offset: one permute serves all layers
+        any_plan.permute(qd, qp)
+        any_plan.permute(kd, kp)
+        any_plan.permute(vd, vp)
+        plans[offs[0]].forward(qp, kp, vp, op)
+        for li, o in enumerate(offs[1:-1]):
+            lq, lk, lv = layer_sets[li % n_sets]
+            plans[o].forward(lq, lk, lv, op)
+        plans[offs[-1]].forward_unpermute(qp, kp, vp, od)
+
+    l0 = hb.launch_count()
+    sched_step()
+    per_step_launches = hb.launch_count() - l0
+    for _ in range(2):
+        sched_step()
+    torch.cuda.synchronize()
+    time.sleep(COOL_DOWN_S)
+    reps = max(3, min(steps, 10))
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record(stream)
+    for _ in range(reps):
+        sched_step()
+    s1.record(stream)
+    torch.cuda.synchronize()
+    sched_ms = s0.elapsed_time(s1) / reps
+    for p_ in plans.values():
+        assert p_.status() == 0, "device-side wait timed out"
+        p_.destroy()
+    assert torch.isfinite(od.float()).all()
+    return {"workload": "%s: %dx%d + %d text, %d heads x %d, tile %d, shared %d" % (
+                wl.name, wl.H, wl.W, wl.n_text, wl.heads, wl.head_dim, wl.tile, wl.shared_region),
+            "layers": SCHEDULE_LAYERS, "distinct_plans": len(plans), "ms_per_step": sched_ms,
+            "ms_per_layer": sched_ms / SCHEDULE_LAYERS, "useful_tflops": sched_flops / (sched_ms * 1e-3) / 1e12,
+            "useful_gflop_per_step": sched_flops / 1e9, "launches_per_step": int(per_step_launches),
+            "offsets": "(layer * tile / 4) mod HW", "reps": reps,
+            "note": "timed: permute(Q), permute(K), permute(V) + 57 forward launches (the last with the exit unpermute "
+                    "fused into its epilogue); the middle layers rotate through %d sets of Q/K/V buffers so that no "
+                    "layer finds its inputs in L2" % n_sets}
 
 
 def main():
@@ -336,15 +462,34 @@ def main():
     torch.cuda.synchronize()
     launches0 = hb.launch_count()
     sampler.start()
+    t_region0 = time.perf_counter()
     start.record(stream)
     for i in range(args.steps):
         step(evs[i], args.warmup + i)
     stop.record(stream)
     torch.cuda.synchronize()
+    t_region1 = time.perf_counter()
+    launches = hb.launch_count() - launches0
+    # SM cycles / nanoseconds the first CTA of the last timed forward launch was resident: the
+    # clock the kernel really ran at (NVML samples are too coarse for a region of a few milliseconds)
+    lc = plan.export(hb.EXPORT_LAUNCH_CLOCK)
+    kernel_clock = {"sm_cycles": int(lc[0]), "ns": int(lc[1]),
+                    "effective_sm_mhz": (1e3 * float(lc[0]) / float(lc[1])) if lc[1] > 0 else None}
+    # The timed region is short; the same steps go on, untimed, until the sampler has seen at
+    # least 0.3 s of this load, so that the clock record has enough samples to mean something.
+    i_extra = 0
+    while time.perf_counter() - t_region0 < 0.3:
+        step(None, args.warmup + args.steps + i_extra)
+        i_extra += 1
+        if i_extra % 8 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
     if distributed:
         dist.barrier()
-    clocks = sampler.stop()
-    launches = hb.launch_count() - launches0
+    clocks = sampler.stop(window=(t_region0, t_region1))
+    clocks["kernel"] = kernel_clock
+    clocks["note"] = ("NVML polled every ms while the timed steps and %d further untimed repeats of the same step ran "
+                      "(>= 0.3 s of load); kernel = SM cycles / ns of one forward launch, read from the kernel" % i_extra)
     total_ms = start.elapsed_time(stop)
     if distributed:
         t = torch.tensor([total_ms], device="cuda")
@@ -364,7 +509,32 @@ def main():
     torch.cuda.synchronize()
     unperm_ms = [ue[i].elapsed_time(ue[i + 1]) for i in range(10)]
     fwd_avg = statistics.mean(fwd_ms)
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    # ---- sustained: forward launches back to back for >= 2 s, with their own clock record
+    sustained = None
+    if world == 1 and not args.no_sustained:
+        smp = ClockSampler(local)
+        n_s = max(50, int(2.2e3 / max(fwd_avg, 1e-3)))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        smp.start()
+        s0.record(stream)
+        for i in range(n_s):
+            a_qp, a_kp, a_vp = sets[i % n_sets][3:6]
+            plan.forward(a_qp, a_kp, a_vp, op)
+        s1.record(stream)
+        torch.cuda.synchronize()
+        s_clk = smp.stop()
+        s_ms = s0.elapsed_time(s1) / n_s
+        lc = plan.export(hb.EXPORT_LAUNCH_CLOCK)
+        s_tf = flops / (s_ms * 1e-3) / 1e12
+        sustained = {"launches": n_s, "seconds": s0.elapsed_time(s1) * 1e-3, "ms_per_call": s_ms, "useful_tflops": s_tf,
+                     "frac_of_measured_sustained_peak": s_tf / peaks["bf16_tflops_sustained"],
+                     "frac_of_measured_burst_peak": s_tf / peaks["bf16_tflops"],
+                     "clocks": s_clk,
+                     "effective_sm_mhz_last_launch": (1e3 * float(lc[0]) / float(lc[1])) if lc[1] > 0 else None}
+    # whole-job work: replicas = one batch per rank, heads = one batch split over the ranks
+    total_flops = 4.0 * wl.head_dim * full_heads * wl.batch * nnz
+    value = total_flops / (ms_per_step * 1e-3) / 1e12
     attn_tflops = flops / (fwd_avg * 1e-3) / 1e12
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
@@ -389,7 +559,7 @@ def main():
             t = torch.tensor([e2e_ms], device="cuda")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e2e_ms = float(t.item())
-        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        e2e = {"value": total_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": 3 * tensor_bytes, "d2h_bytes_per_step": tensor_bytes,
                "api": "hilberta_forward_host (pinned host buffers; per slice of heads: H2D, one launch with entry and exit gathers fused in, D2H; the slices are pipelined over two copy streams)",
                "steps": n_e2e}
@@ -521,52 +691,21 @@ def main():
         plan8.destroy()
         del f_sets, o8
 
+    # free the main workload's extra buffers before the other sizes are measured
+    del sets[1:]
+    torch.cuda.empty_cache()
+
     schedule = None
-    if args.schedule:
-        from paper_2509_26538_b200.inputs import SCHEDULE_LAYERS, schedule_offset
-        offs = [schedule_offset(layer, wl.tile, wl.HW) for layer in range(SCHEDULE_LAYERS)]
-        plans = {}
-        for o in sorted(set(offs)):
-            plans[o] = hb.Plan(wl.H, wl.W, wl.tile, o, wl.shared_region, wl.n_text)
-            plans[o].bind_like(qp)
-        sched_flops = sum(4.0 * wl.head_dim * wl.heads * wl.batch * int(plans[o].export(hb.EXPORT_NNZ)[0])
-                          for o in offs)
+    if world == 1 and (args.schedule or not args.no_configs):
+        schedule = run_schedule57(hb, torch, wl if args.schedule else WORKLOADS["flux1024"], stream, args.steps)
 
-        # every layer of a real step has its own activations: the layers rotate through the
-        # permuted copies of the buffer sets, so a layer does not find its Q, K, V in L2
-        for a_q, a_k, a_v, a_qp, a_kp, a_vp, _ in sets[1:]:
-            plan.permute(a_q, a_qp)
-            plan.permute(a_k, a_kp)
-            plan.permute(a_v, a_vp)
-
-        def sched_step():
-            plan.permute(qd, qp)
-            plan.permute(kd, kp)
-            plan.permute(vd, vp)
-            for li, o in enumerate(offs[:-1]):
-                lq, lk, lv = sets[li % n_sets][3:6]
-                plans[o].forward(lq, lk, lv, op)
-            plans[offs[-1]].forward_unpermute(qp, kp, vp, od)
-
-        for _ in range(3):
-            sched_step()
-        torch.cuda.synchronize()
-        reps = max(3, min(args.steps, 10))
-        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s0.record(stream)
-        for _ in range(reps):
-            sched_step()
-        s1.record(stream)
-        torch.cuda.synchronize()
-        sched_ms = s0.elapsed_time(s1) / reps
-        schedule = {"layers": SCHEDULE_LAYERS, "distinct_plans": len(plans), "ms_per_step": sched_ms,
-                    "ms_per_layer": sched_ms / SCHEDULE_LAYERS, "useful_tflops": sched_flops / (sched_ms * 1e-3) / 1e12,
-                    "offsets": "(layer * tile / 4) mod HW", "reps": reps,
-                    "note": "one entry permute of Q, K, V; the layers rotate through %d sets of Q/K/V buffers; "
-                            "the last layer writes in original order" % n_sets}
-        for p_ in plans.values():
-            assert p_.status() == 0
-            p_.destroy()
+    configs = None
+    if world == 1 and not args.no_configs and not args.groups:
+        configs = {}
+        for name, tiles in (("flux1024", (256, 512, 1024)), ("flux4096", (2048,))):
+            for tile in tiles:
+                c_wl = WORKLOADS[name].with_(tile=tile, layer_offset=tile // 2)
+                configs["%s_tile%d" % (name, tile)] = time_forward_config(hb, torch, c_wl, peaks, stream)
 
     if rank != 0:
         if distributed:
@@ -578,8 +717,8 @@ def main():
         "metric": "sparse-attn useful TFLOP/s at %s (Flux shape)" % {"flux1024": "1024^2", "flux2048": "2048^2",
                                                                       "flux4096": "4096^2"}.get(wl.name, wl.name),
         "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic", "config": workload_config(wl, world),
+        "higher_is_better": True, "scaling": "strong" if shard_heads else "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": workload_config(wl, world, "heads" if shard_heads else "replicas"),
         "attn_ms_per_call": fwd_avg, "attn_ms_per_call_median": statistics.median(fwd_ms),
         "attn_ms_per_call_min": min(fwd_ms), "attn_useful_tflops": attn_tflops,
         "pct_of_nominal_bf16_peak": 100.0 * attn_tflops / NOMINAL_BF16_TFLOPS,
@@ -594,7 +733,7 @@ def main():
                      "unit": "TFLOP/s", "frac": attn_tflops / peak, "peak_source": peaks["source"] + " burst",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "traffic": FORWARD_DRAM_TRAFFIC_BYTES.get(wl.name)},
-        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "fused_step": fused, "backward": backward, "fp8_forward": fp8, "schedule57": schedule,
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "sustained": sustained, "fused_step": fused, "backward": backward, "fp8_forward": fp8, "schedule57": schedule, "configs": configs,
         "context": {"paper": "A100, Triton kernel vs FlashAttention-2: 2.3x at 1024^2, 4.17x at 2048^2 "
                              "(4.36 ms per call at 2048^2, 16 tiles)", "same_gpu": context_rows},
     }
