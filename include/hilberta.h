@@ -185,7 +185,14 @@ int hilberta_plan_bind(hilberta_plan_t *plan, int batch, int heads, int head_dim
  *
  *   q, k, v   device pointers, PHYSICAL token order, layout as bound; read only.
  *   out       device pointer, same layout, written; must not overlap q, k or v.
+ *             The call rejects `out` EQUAL to an input (ERR_INVALID); buffers that overlap
+ *             partly are not detected (with strided, interleaved layouts overlapping
+ *             address ranges are legitimate) and give undefined results.
  *             bf16 and e4m3: all four 16-byte aligned.
+ *   values    q, k and v must be finite over the WHOLE tensors: the tensor-core kernels
+ *             multiply the rows of a partly masked 128-key block by weights that are
+ *             exactly zero, and 0 * Inf or 0 * NaN in a token the mask excludes would
+ *             reach rows that must not see it.
  *   plan      a bound plan.
  *   stream    the launch is asynchronous on this stream; no allocation, no
  *             synchronisation.
@@ -223,8 +230,9 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  * carries lse * log2(e) and delta between the launches, so two backward calls on
  * the same plan must not overlap on the device.
  *
- * Errors: ERR_INVALID (NULL, misaligned or aliasing pointers, wrong device),
- * ERR_UNBOUND, ERR_CUDA. */
+ * Errors: ERR_INVALID (NULL or misaligned pointers, an output equal to another
+ * argument, wrong device), ERR_UNBOUND, ERR_CUDA.  Partly overlapping buffers are
+ * not detected (see hilberta_forward). */
 int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                       const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
                       void *stream);
@@ -238,7 +246,11 @@ int hilberta_backward(const void *dout, const void *q, const void *k, const void
  * memory to its own pool at start-up, so that a later cudaMalloc fails; a
  * latency-bound loop that must avoid the device-wide synchronisation an
  * allocation implies; a process that keeps dozens of bound plans (one per layer
- * offset) and does not want a scratch array in each.  This variant puts the
+ * offset) and wants them to share one scratch array at call time.  (hilberta_plan_bind
+ * itself still allocates: the plan's work lists, schedules and its own per-plan
+ * scratch.  Build and bind every plan first, before device memory is handed to the
+ * host application's pool; only the calls made afterwards are allocation-free.)
+ * This variant puts the
  * scratch in one fixed array of HILBERTA_STATIC_SCRATCH_FLOATS floats (4 MiB)
  * that is part of the library image: every GPU that loads the library holds it
  * until the process exits, and every plan and every call shares it.
@@ -317,6 +329,17 @@ int hilberta_forward_host(const void *q, const void *k, const void *v, void *out
  * inside the kernel gave up (the output is then undefined).  Synchronises the
  * device.  Clears the flag. */
 int hilberta_plan_status(hilberta_plan_t *plan);
+
+/* Host-side check of a kernel work list (no GPU involved; hilberta_plan_bind runs it on every
+ * list it builds and fails with ERR_INVALID rather than upload a bad one).  The attention kernels
+ * read the query rows and key ranges of their work items unchecked, so this is what stands
+ * between a planning bug and an out-of-range access.  items: n_items records of ten int32:
+ * q_start, q_rows, n_seg, seg_start[3], seg_len[3], kv_blocks.  Returns HILBERTA_OK iff every
+ * item has 1 <= q_rows <= item_rows and its rows inside [0, S); 1 <= n_seg <= 3 key ranges, each
+ * non-empty and inside [0, S), pairwise disjoint; kv_blocks = sum of ceil(seg_len / block); and the
+ * items' query ranges cover [0, S) exactly once.  Otherwise ERR_INVALID.  (Sec. 3.2 / 3.3: every
+ * query row belongs to the prefix or to exactly one slid tile.) */
+int hilberta_check_work_list(const int32_t *items, int n_items, int S, int item_rows, int block);
 
 /* Failure-detection self-test: launches a one-warp kernel that waits, with a 1 ms
  * deadline, on a barrier nothing arrives on -- the same bounded wait every role of

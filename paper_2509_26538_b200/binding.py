@@ -30,6 +30,7 @@ SYMBOLS = (
     "hilberta_backward_static", "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
+    "hilberta_check_work_list",
     "hilberta_plan_status", "hilberta_selftest_timeout", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
     "hilberta_last_cuda_error",
 )
@@ -87,6 +88,8 @@ def lib():
         f = getattr(L, name)
         f.argtypes = [vp, vp, vp, i32, i32, i32, vp]
         f.restype = i32
+    L.hilberta_check_work_list.argtypes = [vp, i32, i32, i32, i32]
+    L.hilberta_check_work_list.restype = i32
     L.hilberta_selftest_timeout.argtypes = [vp, vp]
     L.hilberta_selftest_timeout.restype = i32
     L.hilberta_plan_status.argtypes = [vp]
@@ -101,6 +104,12 @@ def lib():
     L.hilberta_last_cuda_error.restype = i32
     _lib = L
     return L
+
+
+def check_work_list(items, S: int, item_rows: int, block: int) -> int:
+    """Status of hilberta_check_work_list for an [n, 10] int32 array of work items (host only)."""
+    a = np.ascontiguousarray(items, dtype=np.int32).reshape(-1, 10)
+    return int(lib().hilberta_check_work_list(a.ctypes.data, a.shape[0], int(S), int(item_rows), int(block)))
 
 
 def _check(status: int, where: str):

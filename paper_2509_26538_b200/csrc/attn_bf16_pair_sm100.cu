@@ -637,6 +637,10 @@ int attn_bf16_pair_prepare(hilberta_plan_t *p) {
     if (max_pairs < 1) return HILBERTA_OK;
     auto cost_of = [](const WorkItem &it) { return (long long)it.kv_blocks * 10 + 6; };
     std::vector<WorkItem> items = build_work_items(p, ITEM_ROWS, BN);
+    {
+        const int rc_items = check_work_items(items.data(), (int)items.size(), p->S, ITEM_ROWS, BN);
+        if (rc_items != HILBERTA_OK) return rc_items;
+    }
     if (items.empty()) return HILBERTA_OK;
     std::stable_sort(items.begin(), items.end(),
                      [&](const WorkItem &a, const WorkItem &b) { return cost_of(a) > cost_of(b); });

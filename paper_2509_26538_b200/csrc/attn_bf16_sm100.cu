@@ -755,6 +755,10 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
     // blocks take about 1.3 x half the time of a two-tile unit's (costs in tenths of a tile-block)
     auto cost_of = [](const WorkItem &it) { return (long long)it.kv_blocks * (it.q_rows > BM ? 20 : 13) + 20; };
     std::vector<WorkItem> items = build_work_items(p, ITEM_ROWS, BN);
+    {
+        const int rc_items = check_work_items(items.data(), (int)items.size(), p->S, ITEM_ROWS, BN);
+        if (rc_items != HILBERTA_OK) return rc_items;
+    }
     std::stable_sort(items.begin(), items.end(),
                      [&](const WorkItem &a, const WorkItem &b) { return cost_of(a) > cost_of(b); });
     std::vector<long long> cost;

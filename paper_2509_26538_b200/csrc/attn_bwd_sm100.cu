@@ -571,6 +571,10 @@ delta_kernel(const __nv_bfloat16 *__restrict__ dout, const __nv_bfloat16 *__rest
 // Also allocates the per-row scratch: lse * log2 e for every row, then delta for every row.  Called from hilberta_plan_bind for bf16 bindings.
 int attn_bwd_prepare(hilberta_plan_t *p) {
     std::vector<WorkItem> items = build_work_items(p, BM, BK);
+    {
+        const int rc_items = check_work_items(items.data(), (int)items.size(), p->S, BM, BK);
+        if (rc_items != HILBERTA_OK) return rc_items;
+    }
     std::stable_sort(items.begin(), items.end(),
                      [](const WorkItem &a, const WorkItem &b) { return a.kv_blocks > b.kv_blocks; });
     std::vector<long long> cost;

@@ -131,6 +131,8 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
 // schedule.cu: work lists (runs of item_rows rows with their up to three key ranges, counted in
 // blocks of `block` rows) and the static longest-first assignment of (item, batch * head) units to CTAs
 std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, int block);
+// HILBERTA_OK iff the list is safe to hand to a kernel (ranges inside [0, S), rows covered exactly once)
+int check_work_items(const WorkItem *items, int n, int S, int item_rows, int block);
 int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
                     WorkUnit **d_units, int **d_cta_begin, int *n_cta_out);
 int attn_bf16_prepare(hilberta_plan_t *p);

@@ -52,6 +52,40 @@ std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, 
     return items;
 }
 
+// Every kernel reads the key ranges and query rows of its work items without further checks, so the
+// lists are validated on the host before anything is uploaded: each item's rows and key ranges lie
+// inside [0, S), its key ranges do not overlap, its block count matches them, and the items' query
+// ranges cover [0, S) exactly once.
+int check_work_items(const WorkItem *items, int n, int S, int item_rows, int block) {
+    if (n < 0 || S < 0 || item_rows < 1 || block < 1 || (n > 0 && !items)) return HILBERTA_ERR_INVALID;
+    std::vector<std::pair<int, int>> rows;   // (q_start, q_rows)
+    rows.reserve((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        const WorkItem &it = items[i];
+        if (it.q_rows < 1 || it.q_rows > item_rows || it.q_start < 0 || it.q_start > S - it.q_rows)
+            return HILBERTA_ERR_INVALID;
+        if (it.n_seg < 1 || it.n_seg > 3) return HILBERTA_ERR_INVALID;
+        long long blocks = 0;
+        for (int a = 0; a < it.n_seg; ++a) {
+            if (it.seg_len[a] < 1 || it.seg_start[a] < 0 || it.seg_start[a] > S - it.seg_len[a])
+                return HILBERTA_ERR_INVALID;
+            blocks += (it.seg_len[a] + block - 1) / block;
+            for (int b = 0; b < a; ++b)
+                if (it.seg_start[a] < it.seg_start[b] + it.seg_len[b] && it.seg_start[b] < it.seg_start[a] + it.seg_len[a])
+                    return HILBERTA_ERR_INVALID;   // a key would be counted twice
+        }
+        if (blocks != it.kv_blocks) return HILBERTA_ERR_INVALID;
+        rows.push_back(std::make_pair(it.q_start, it.q_rows));
+    }
+    std::sort(rows.begin(), rows.end());
+    int next = 0;
+    for (const std::pair<int, int> &r : rows) {
+        if (r.first != next) return HILBERTA_ERR_INVALID;   // a gap or an overlap between items
+        next = r.first + r.second;
+    }
+    return next == S ? HILBERTA_OK : HILBERTA_ERR_INVALID;
+}
+
 // items must be sorted by descending cost.  On success *d_units holds items.size() * bh units
 // grouped by CTA and *d_cta_begin the n_cta + 1 offsets (both device memory, owned by the caller).
 int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
@@ -88,3 +122,9 @@ int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long l
 }
 
 }  // namespace hilberta
+
+static_assert(sizeof(hilberta::WorkItem) == 10 * sizeof(int32_t), "hilberta_check_work_list takes ten ints per item");
+
+extern "C" int hilberta_check_work_list(const int32_t *items, int n_items, int S, int item_rows, int block) {
+    return hilberta::check_work_items(reinterpret_cast<const hilberta::WorkItem *>(items), n_items, S, item_rows, block);
+}

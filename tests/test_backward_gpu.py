@@ -115,7 +115,7 @@ def test_backward_argument_checks():
 
 def test_backward_flux2048_sampled():
     """Bench launch configuration (24 heads, 128x128 + 512 tokens); the oracle computes sampled
-    dq rows and dk / dv columns of two heads one by one."""
+    dq rows and dk / dv columns of every head one by one."""
     from paper_2509_26538_b200.inputs import WORKLOADS, make_qkv, sample_rows
     wl = WORKLOADS["flux2048"]
     q, k, v = make_qkv(wl)
@@ -149,7 +149,7 @@ def test_backward_flux2048_sampled():
                 edge += [int(p2o[s]), int(p2o[s + n - 1]), int(p2o[s + min(n - 1, 63)]), int(p2o[s + min(n - 1, 64)])]
     toks = np.array(sorted(set(sample_rows(wl, 40) + edge)), dtype=np.int32)
     ig, grp = orc.token_classes(wl.H, wl.W, wl.tile, wl.layer_offset, wl.shared_region, wl.n_text)
-    for h in (0, wl.heads - 1):
+    for h in range(wl.heads):
         sl = lambda t: t[:, h:h + 1].float().numpy()
         ref = attn_c.attention_backward(sl(q), sl(k), sl(v), sl(do), ig, grp, rows=toks, cols=toks)
         for name, gt, r in zip(("dq", "dk", "dv"), got, ref):

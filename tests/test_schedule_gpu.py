@@ -1,6 +1,7 @@
 """Full per-step layer schedule at 1024^2 (57 layers, offsets (layer * tile / 4) mod HW),
 with the entry and exit gathers: plans per distinct offset are bit-exact, and the
-forward of sampled layers matches the oracle on sampled rows of every head."""
+forward matches the oracle over the WHOLE output tensor (all 4608 tokens, all 24 heads) for a layer of
+each of the four distinct masks, and on sampled rows for later layers, all run through the schedule's own loop."""
 import numpy as np
 import pytest
 import torch
@@ -41,16 +42,24 @@ def test_schedule_57_layers():
         for p in plans.values():
             p.bind_like(qp)
         rows = sample_rows(wl, 48)
-        check_layers = {0, 1, 2, 3, 17, 56}
+        whole_layers = {0, 1, 2, 3}          # offsets 0, 256, 512, 768: the four masks
+        sampled_layers = {17, 38, 56}
+        qf, kf, vf = (t.float().numpy() for t in (q, k, v))
         for layer, o in enumerate(offsets):
             plans[o].forward(qp, kp, vp, op)
-            if layer in check_layers:
+            if layer in whole_layers or layer in sampled_layers:
                 first.unpermute(op, od)
                 torch.cuda.synchronize()
-                got = od[:, :, rows].cpu().double().numpy()
                 ig, grp = orc.token_classes(wl.H, wl.W, tile, o, wl.shared_region, wl.n_text)
-                ref = attn_c.attention_rows(q.float().numpy(), k.float().numpy(), v.float().numpy(), ig, grp, rows=rows)
+                if layer in whole_layers:
+                    got = od.cpu().double().numpy()
+                    ref = attn_c.attention_rows(qf, kf, vf, ig, grp)
+                else:
+                    got = od[:, :, rows].cpu().double().numpy()
+                    ref = attn_c.attention_rows(qf, kf, vf, ig, grp, rows=rows)
+                assert np.isfinite(got).all()
                 assert orc.max_abs_err(got, ref) <= 1e-2 and orc.rel_l2_err(got, ref) <= 5e-3, (layer, o)
+        assert len({offsets[l] % tile for l in whole_layers}) == 4
         for p in plans.values():
             assert p.status() == 0
     finally:

@@ -22,10 +22,10 @@ from paper_2509_26538_b200 import binding as hb
 pytestmark = pytest.mark.gpu
 
 
-def _problem(H, W, tile, o, hs, nt, B, heads, seed):
+def _problem(H, W, tile, o, hs, nt, B, heads, seed, dtype=torch.bfloat16, D=128):
     S = nt + H * W
     g = torch.Generator().manual_seed(seed)
-    qp, kp, vp, dop = (torch.randn((B, heads, S, 128), generator=g).to(torch.bfloat16).cuda() for _ in range(4))
+    qp, kp, vp, dop = (torch.randn((B, heads, S, D), generator=g).to(dtype).cuda() for _ in range(4))
     plan = hb.Plan(H, W, tile, o, hs, nt)
     plan.bind_like(qp)
     out = torch.empty_like(qp)
@@ -53,8 +53,59 @@ def test_static_scratch_backward_matches_plan_scratch_backward_twice():
                 assert _rel_l2(g, w) <= 5e-3, (name, _rel_l2(g, w))
                 scale = max(1.0, float(w.float().abs().max()))
                 assert float((g.float() - w.float()).abs().max()) <= 1e-2 * scale, name
+                # the two entry points run the same kernels on the same inputs and differ only in
+                # where the scratch lives: the results are the same bits
+                assert torch.equal(g.view(torch.int16), w.view(torch.int16)), name
         finally:
             plan.destroy()
+
+
+def test_static_scratch_backward_allocates_no_device_memory():
+    """After the first call on a device (which looks up the array's address) a call must leave the
+    amount of free device memory exactly as it found it."""
+    plan, args = _problem(32, 32, 256, 128, 4, 77, 1, 3, 13)
+    try:
+        got = [torch.empty_like(args[1]) for _ in range(3)]
+        plan.backward_static(*args, *got)          # first call: set-up
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        for _ in range(3):
+            plan.backward_static(*args, *got)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert plan.status() == 0
+        assert free1 == free0, (free0, free1)
+    finally:
+        plan.destroy()
+
+
+def test_static_scratch_backward_fp32_binding():
+    plan, args = _problem(16, 16, 64, 16, 2, 24, 1, 2, 14, dtype=torch.float32, D=64)
+    try:
+        want = [torch.empty_like(args[1]) for _ in range(3)]
+        plan.backward(*args, *want)
+        got = [torch.full_like(args[1], float("nan")) for _ in range(3)]
+        plan.backward_static(*args, *got)
+        assert plan.status() == 0
+        for name, g, w in zip(("dq", "dk", "dv"), got, want):
+            assert torch.equal(g.view(torch.int32), w.view(torch.int32)), name
+    finally:
+        plan.destroy()
+
+
+def test_static_scratch_backward_accepts_the_exact_fit():
+    """2 * batch * heads * S == 2^20 floats fills the array exactly: still accepted, results the same bits."""
+    plan, args = _problem(32, 32, 256, 0, 0, 0, 8, 64, 15)      # S = 1024, batch * heads = 512
+    try:
+        want = [torch.empty_like(args[1]) for _ in range(3)]
+        plan.backward(*args, *want)
+        got = [torch.full_like(args[1], float("nan")) for _ in range(3)]
+        plan.backward_static(*args, *got)
+        assert plan.status() == 0
+        for name, g, w in zip(("dq", "dk", "dv"), got, want):
+            assert torch.equal(g.view(torch.int16), w.view(torch.int16)), name
+    finally:
+        plan.destroy()
 
 
 def test_static_scratch_backward_rejects_what_does_not_fit():
