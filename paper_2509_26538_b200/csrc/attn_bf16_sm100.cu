@@ -182,6 +182,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __shared__ int abort_flag;
     __shared__ long long stamp[2];
     static_assert(!FP8 || HD == 128, "e4m3 operands: head dim 128 only");
+#ifdef HB_STAMPS
+    if (threadIdx.x == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        prm.status[1024 + 4 * blockIdx.x] = (int)(ns & 0x7fffffff);
+    }
+#endif
     constexpr int TILE_BYTES = tile_bytes(HD, FP8);
     constexpr int NSLAB = TILE_BYTES / SLAB_BYTES;
     using elem_t = typename std::conditional<FP8, uint8_t, __nv_bfloat16>::type;
@@ -266,16 +273,52 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             const WorkItem wi = prm.work[unit.item];
             const long long bh_off = (long long)(unit.bh / prm.heads) * prm.stride_b +
                                      (long long)(unit.bh % prm.heads) * prm.stride_h;
-            const int nt = wi.q_rows > BM ? 2 : 1;
+            const bool dual = unit.bh2 >= 0;   // the item for two heads, one per query-tile slot
+            const long long bh_off2 = !dual ? bh_off
+                                            : (long long)(unit.bh2 / prm.heads) * prm.stride_b +
+                                                  (long long)(unit.bh2 % prm.heads) * prm.stride_h;
+            const int nt = (dual || wi.q_rows > BM) ? 2 : 1;
             ok = wait_or_abort(bar(Q_EMPTY), (qc & 1) ^ 1, &abort_flag, prm.status, 0x111);
             if (!ok) break;
             ++qc;
             for (int t = 0; t < nt; ++t) {
                 int ia, ib;
-                load_rows(wi.q_start + t * BM, ia, ib);
-                copy_tile(sQ + t * TILE_BYTES, (const elem_t *)prm.gq + bh_off, ia, ib);
+                load_rows(wi.q_start + (dual ? 0 : t * BM), ia, ib);
+                copy_tile(sQ + t * TILE_BYTES, (const elem_t *)prm.gq + (t ? bh_off2 : bh_off), ia, ib);
             }
             publish(bar(Q_FULL));
+            if (dual) {
+                // two K/V streams (same rows, two heads), entries in the order the MMA issuer uses them:
+                // K_0(0) K_1(0), then per block V_0(j) K_0(j+1) V_1(j) K_1(j+1)
+                auto emit = [&](const void *g, long long off, int ia, int ib) {
+                    const uint32_t sl = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
+                    ++kvc;
+                    if (!wait_or_abort(bar(KV_EMPTY + sl), ph ^ 1, &abort_flag, prm.status, 0x112)) return false;
+                    copy_tile(sKV + sl * TILE_BYTES, (const elem_t *)g + off, ia, ib);
+                    publish(bar(KV_FULL + sl));
+                    return true;
+                };
+                int ia, ib;
+                load_rows(wi.seg_start[0], ia, ib);
+                ok = emit(prm.gk, bh_off, ia, ib) && emit(prm.gk, bh_off2, ia, ib);
+                for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
+                    const int nb = item_blocks(wi, seg);
+                    for (int j = 0; ok && j < nb; ++j) {
+                        int row_n = -1;
+                        if (j + 1 < nb) row_n = wi.seg_start[seg] + (j + 1) * BN;
+                        else if (seg + 1 < wi.n_seg) row_n = wi.seg_start[seg + 1];
+                        int na = -1, nbi = -1;
+                        if (row_n >= 0) load_rows(row_n, na, nbi);
+                        ok = emit(prm.gv, bh_off, ia, ib);
+                        if (row_n >= 0) ok = ok && emit(prm.gk, bh_off, na, nbi);
+                        ok = ok && emit(prm.gv, bh_off2, ia, ib);
+                        if (row_n >= 0) ok = ok && emit(prm.gk, bh_off2, na, nbi);
+                        ia = na;
+                        ib = nbi;
+                    }
+                }
+                continue;
+            }
             for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                 const int nb = item_blocks(wi, seg);
                 for (int j = 0; ok && j < nb; ++j) {
@@ -321,12 +364,25 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             prefetch_tmap(&tmV);
             uint32_t kvc = 0, qc = 0;
             bool ok = true;
+            // one ring entry: the K or V tile at key row `row` of head (h, b)
+            auto emit = [&](const CUtensorMap *tm, int row, int h, int b) {
+                const uint32_t s = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
+                ++kvc;
+                if (!wait_or_abort(bar(KV_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x102)) return false;
+                mbar_expect_tx(bar(KV_FULL + s), TILE_BYTES);
+#pragma unroll
+                for (int sl = 0; sl < NSLAB; ++sl)
+                    tma_load_4d(sKV + s * TILE_BYTES + sl * SLAB_BYTES, tm, bar(KV_FULL + s), 64 * sl, row, h, b);
+                return true;
+            };
             for (int u = u_begin; ok && u < u_end; ++u) {
                 const WorkUnit unit = prm.units[u];
                 const WorkItem wi = prm.work[unit.item];
                 const int bh = unit.bh;
                 const int b = bh / prm.heads, h = bh % prm.heads;
-                const int nt = wi.q_rows > BM ? 2 : 1;
+                const bool dual = unit.bh2 >= 0;   // the item for two heads, one per query-tile slot
+                const int b2 = dual ? unit.bh2 / prm.heads : b, h2 = dual ? unit.bh2 % prm.heads : h;
+                const int nt = (dual || wi.q_rows > BM) ? 2 : 1;
                 ok = wait_or_abort(bar(Q_EMPTY), (qc & 1) ^ 1, &abort_flag, prm.status, 0x101);
                 if (!ok) break;
                 ++qc;
@@ -335,24 +391,30 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                     for (int sl = 0; sl < NSLAB; ++sl)
                         tma_load_4d(sQ + t * TILE_BYTES + sl * SLAB_BYTES, &tmQ, bar(Q_FULL), 64 * sl,
-                                    wi.q_start + t * BM, h, b);
+                                    wi.q_start + (dual ? 0 : t * BM), t ? h2 : h, t ? b2 : b);
                 }
+                // Ring entries in the order the MMA issuer consumes them.  One stream (both tiles read
+                // the same tiles): K(0) V(0) K(1) V(1) ...  Two streams: K_0(0) K_1(0), then per block
+                // V_0(j) K_0(j+1) V_1(j) K_1(j+1).
+                bool first_block = true;
                 for (int seg = 0; ok && seg < wi.n_seg; ++seg) {
                     const int nb = item_blocks(wi, seg);
-                    for (int j = 0; j < nb; ++j) {
+                    for (int j = 0; ok && j < nb; ++j) {
                         const int row = wi.seg_start[seg] + j * BN;
-#pragma unroll
-                        for (int kv = 0; kv < 2; ++kv, ++kvc) {
-                            const uint32_t s = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
-                            ok = wait_or_abort(bar(KV_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x102);
-                            if (!ok) break;
-                            const CUtensorMap *tm = kv ? &tmV : &tmK;
-                            mbar_expect_tx(bar(KV_FULL + s), TILE_BYTES);
-#pragma unroll
-                            for (int sl = 0; sl < NSLAB; ++sl)
-                                tma_load_4d(sKV + s * TILE_BYTES + sl * SLAB_BYTES, tm, bar(KV_FULL + s), 64 * sl, row, h, b);
+                        if (!dual) {
+                            ok = emit(&tmK, row, h, b) && emit(&tmV, row, h, b);
+                        } else {
+                            // the next block's key row, if there is one
+                            int row_n = -1;
+                            if (j + 1 < nb) row_n = row + BN;
+                            else if (seg + 1 < wi.n_seg) row_n = wi.seg_start[seg + 1];
+                            if (first_block) ok = emit(&tmK, row, h, b) && emit(&tmK, row, h2, b2);
+                            first_block = false;
+                            ok = ok && emit(&tmV, row, h, b);
+                            if (row_n >= 0) ok = ok && emit(&tmK, row_n, h, b);
+                            ok = ok && emit(&tmV, row, h2, b2);
+                            if (row_n >= 0) ok = ok && emit(&tmK, row_n, h2, b2);
                         }
-                        if (!ok) break;
                     }
                 }
             }
@@ -366,7 +428,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     } else if (warp == 9) {
         // ---------------------------------------------------------- MMA issuer
         if (elect_one()) {
-            uint32_t g = 0;   // blocks consumed so far: K of block g is ring entry 2g, V is 2g + 1
+            uint32_t ent = 0;   // ring entries consumed so far (the producer fills them in the order they are used here)
             uint32_t qc = 0;
             uint32_t cP[QT] = {0, 0};
             bool ok = true;
@@ -375,28 +437,95 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #endif
             auto slot_of = [](uint32_t e) { return e % NSTAGE; };
             auto phase_of = [](uint32_t e) { return (e / NSTAGE) & 1; };
+            // O_t (+)= P_t V for block j of tile t (P arrives in two halves so the first four MMAs overlap
+            // the rest of the softmax), then S_t = Q_t K^T for the next block if there is one
+            auto tile_turn = [&](int t, uint32_t eV, uint32_t eKn, bool accumulate, bool more) {
+#ifdef HB_TIMING
+                const long long tp0 = clock64();
+#endif
+                if (!wait_or_abort(bar(P_READY + t * 2), cP[t] & 1, &abort_flag, prm.status, 0x205 + t)) return false;
+                tc_fence_after();
+#ifdef HB_TIMING
+                tm_p += clock64() - tp0;
+#endif
+                issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, accumulate);
+#ifdef HB_TIMING
+                const long long tp1 = clock64();
+#endif
+                if (!wait_or_abort(bar(P_READY + t * 2 + 1), cP[t] & 1, &abort_flag, prm.status, 0x205 + t)) return false;
+                ++cP[t];
+#ifdef HB_TIMING
+                tm_p += clock64() - tp1;
+#endif
+                tc_fence_after();
+                issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
+                mma_commit(bar(PV_DONE + t));
+                if (more) {
+                    issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
+                    mma_commit(bar(S_FULL + t));
+                }
+                return true;
+            };
             for (int u = u_begin; ok && u < u_end; ++u) {
-                const WorkItem wi = prm.work[prm.units[u].item];
-                const int nt = wi.q_rows > BM ? 2 : 1;
+                const WorkUnit unit = prm.units[u];
+                const WorkItem wi = prm.work[unit.item];
+                const bool dual = unit.bh2 >= 0;
+                const int nt = (dual || wi.q_rows > BM) ? 2 : 1;
                 const int n = wi.kv_blocks;
                 ok = wait_or_abort(bar(Q_FULL), qc & 1, &abort_flag, prm.status, 0x201);
                 if (!ok) break;
                 ++qc;
                 // tiles written by cp.async (generic proxy) are read by the tensor core (async proxy)
                 if (GATHER) fence_proxy_async_smem();
+                if (dual) {
+                    // two K/V streams, one per tile: every ring entry serves one tile and is released as
+                    // soon as the MMAs that read it are issued
+                    for (int t = 0; t < 2; ++t, ++ent) {
+                        ok = wait_or_abort(bar(KV_FULL + slot_of(ent)), phase_of(ent), &abort_flag, prm.status, 0x202);
+                        if (!ok) break;
+                        if (GATHER) fence_proxy_async_smem();
+                        tc_fence_after();
+                        issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(ent) * TILE_BYTES);
+                        mma_commit(bar(S_FULL + t));
+                        mma_commit(bar(KV_EMPTY + slot_of(ent)));
+                    }
+                    if (!ok) break;
+                    if (n == 1) mma_commit(bar(Q_EMPTY));
+                    for (int j = 0; ok && j < n; ++j) {
+                        const bool more = j + 1 < n;
+                        for (int t = 0; t < 2; ++t) {
+                            const uint32_t eV = ent, eKn = ent + 1;
+                            ent += more ? 2 : 1;
+                            ok = wait_or_abort(bar(KV_FULL + slot_of(eV)), phase_of(eV), &abort_flag, prm.status, 0x204);
+                            if (!ok) break;
+                            if (more) {
+                                ok = wait_or_abort(bar(KV_FULL + slot_of(eKn)), phase_of(eKn), &abort_flag, prm.status, 0x203);
+                                if (!ok) break;
+                            }
+                            if (GATHER) fence_proxy_async_smem();
+                            ok = tile_turn(t, eV, eKn, j > 0, more);
+                            if (!ok) break;
+                            mma_commit(bar(KV_EMPTY + slot_of(eV)));
+                            if (more) mma_commit(bar(KV_EMPTY + slot_of(eKn)));
+                        }
+                        if (ok && j + 2 == n) mma_commit(bar(Q_EMPTY));
+                    }
+                    continue;
+                }
+                // one K/V stream: K of block j is entry ent + 2 j, V is ent + 2 j + 1
                 // S_t(0)
-                ok = wait_or_abort(bar(KV_FULL + slot_of(2 * g)), phase_of(2 * g), &abort_flag, prm.status, 0x202);
+                ok = wait_or_abort(bar(KV_FULL + slot_of(ent)), phase_of(ent), &abort_flag, prm.status, 0x202);
                 if (!ok) break;
                 if (GATHER) fence_proxy_async_smem();
                 tc_fence_after();
                 for (int t = 0; t < nt; ++t) {
-                    issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(2 * g) * TILE_BYTES);
+                    issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(ent) * TILE_BYTES);
                     mma_commit(bar(S_FULL + t));
                 }
-                mma_commit(bar(KV_EMPTY + slot_of(2 * g)));
+                mma_commit(bar(KV_EMPTY + slot_of(ent)));
                 if (n == 1) mma_commit(bar(Q_EMPTY));
-                for (int j = 0; j < n; ++j, ++g) {
-                    const uint32_t eV = 2 * g + 1, eKn = 2 * g + 2;
+                for (int j = 0; j < n; ++j, ent += 2) {
+                    const uint32_t eV = ent + 1, eKn = ent + 2;
                     const bool more = j + 1 < n;
 #ifdef HB_TIMING
                     const long long tk0 = clock64();
@@ -411,35 +540,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef HB_TIMING
                     tm_kv += clock64() - tk0;
 #endif
-                    for (int t = 0; t < nt; ++t) {
-#ifdef HB_TIMING
-                        const long long tp0 = clock64();
-#endif
-                        // P arrives in two halves so the first four MMAs overlap the rest of the softmax
-                        ok = wait_or_abort(bar(P_READY + t * 2), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
-                        if (!ok) break;
-                        tc_fence_after();
-#ifdef HB_TIMING
-                        tm_p += clock64() - tp0;
-#endif
-                        issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, j > 0);
-#ifdef HB_TIMING
-                        const long long tp1 = clock64();
-#endif
-                        ok = wait_or_abort(bar(P_READY + t * 2 + 1), cP[t] & 1, &abort_flag, prm.status, 0x205 + t);
-                        if (!ok) break;
-                        ++cP[t];
-#ifdef HB_TIMING
-                        tm_p += clock64() - tp1;
-#endif
-                        tc_fence_after();
-                        issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
-                        mma_commit(bar(PV_DONE + t));
-                        if (more) {
-                            issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
-                            mma_commit(bar(S_FULL + t));
-                        }
-                    }
+                    for (int t = 0; ok && t < nt; ++t) ok = tile_turn(t, eV, eKn, j > 0, more);
                     if (!ok) break;
                     mma_commit(bar(KV_EMPTY + slot_of(eV)));
                     if (more) {
@@ -470,14 +571,25 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const float scale_log2 = prm.scale_log2;
         uint32_t cS = 0, cPV = 0;
         bool ok = true;
+#ifdef HB_STAMPS
+        int st_b2 = 0, st_b1 = 0, st_items2 = 0, st_items1 = 0, st_prefix_blocks = 0;
+#endif
 #ifdef HB_TIMING
         long long tm_wait = 0, tm_soft = 0, tm_epi = 0, tm_mark = clock64(), tm_blocks = 0;
 #endif
         for (int u = u_begin; ok && u < u_end; ++u) {
             const WorkUnit unit = prm.units[u];
             const WorkItem wi = prm.work[unit.item];
-            if (wi.q_rows <= t * BM) continue;  // this tile is absent from the item
-            const int bh = unit.bh;
+#ifdef HB_STAMPS
+            const long long st_unit_t0 = clock64();
+            if (tid == 0) {
+                if (wi.q_rows > BM) { st_b2 += wi.kv_blocks; ++st_items2; } else { st_b1 += wi.kv_blocks; ++st_items1; }
+                if (wi.n_seg == 1) st_prefix_blocks += wi.kv_blocks;
+            }
+#endif
+            const bool dual = unit.bh2 >= 0;   // the item for two heads: tile slot 1 holds the same rows of head bh2
+            if (wi.q_rows <= t * BM && !dual) continue;  // this tile is absent from the item
+            const int bh = (dual && t) ? unit.bh2 : unit.bh;
             const int b = bh / prm.heads, h = bh % prm.heads;
             float m_ref = 0.f, l = 0.f;
             float l_fix = 0.f;   // rounding errors of the blocks' largest weights: part of the output's normaliser, not of lse
@@ -617,7 +729,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             const float inv = 1.f / (l + l_fix);
-            const int row = t * BM + r;
+            const int row = dual ? r : t * BM + r;
             // each thread stores its own row, so writing it at its ORIGINAL position instead
             // of the physical one (the exit gather of Sec. 3.4 fused in) costs one index read
             int out_row = wi.q_start + row;
@@ -655,7 +767,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef HB_TIMING
             { const long long now = clock64(); tm_epi += now - tm_mark; tm_mark = now; }
 #endif
+#ifdef HB_STAMPS
+            if (tid == 0 && blockIdx.x % 5 == 4 && blockIdx.x / 5 < 32 && u - u_begin < 16) {
+                int *w = prm.status + 3072 + (blockIdx.x / 5) * 32 + (u - u_begin) * 2;
+                w[0] = wi.kv_blocks | ((wi.q_rows > BM ? 2 : 1) << 16) | ((wi.n_seg == 1 ? 1 : 0) << 20) | (1 << 24);
+                w[1] = (int)(clock64() - st_unit_t0);
+            }
+#endif
         }
+#ifdef HB_STAMPS
+        if (tid == 0) {
+            int *w = prm.status + 2048 + 8 * blockIdx.x;
+            w[0] = st_b2; w[1] = st_b1; w[2] = st_items2; w[3] = st_items1; w[4] = st_prefix_blocks;
+        }
+#endif
 #ifdef HB_TIMING
         if ((tid & 127) == 0) {
             atomicAdd(prm.status + 8 + t * 4 + 0, (int)(tm_wait >> 4));
@@ -679,6 +804,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
     }
+#ifdef HB_STAMPS
+    if (threadIdx.x == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        prm.status[1024 + 4 * blockIdx.x + 1] = (int)(ns & 0x7fffffff);
+        prm.status[1024 + 4 * blockIdx.x + 2] = (int)(stamp[1] & 0x7fffffff);
+    }
+#endif
 }
 
 // Exercises the bounded wait on purpose: one warp waits, with a 1 ms deadline, on a
@@ -751,9 +884,12 @@ int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
 
 // Work list (items of two query tiles, key blocks of 128) and the static schedules.
 int attn_bf16_prepare(hilberta_plan_t *p) {
-    // a unit with one query tile has no second tile to overlap its softmax with the MMAs: its
-    // blocks take about 1.3 x half the time of a two-tile unit's (costs in tenths of a tile-block)
-    auto cost_of = [](const WorkItem &it) { return (long long)it.kv_blocks * (it.q_rows > BM ? 20 : 13) + 20; };
+    // Cost of a unit in twentieths of a two-tile key block (about 140 SM cycles), from per-unit cycle
+    // counts of the kernel at 1024^2 and 2048^2: two tiles 2760 cycles per block + 5500; one tile --
+    // nothing to overlap its softmax with the MMAs -- 2580 per block + 2600, i.e. hardly cheaper.
+    auto cost_of = [](const WorkItem &it) {
+        return it.q_rows > BM ? (long long)it.kv_blocks * 20 + 40 : (long long)it.kv_blocks * 19 + 20;
+    };
     std::vector<WorkItem> items = build_work_items(p, ITEM_ROWS, BN);
     {
         const int rc_items = check_work_items(items.data(), (int)items.size(), p->S, ITEM_ROWS, BN);
@@ -761,8 +897,14 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
     }
     std::stable_sort(items.begin(), items.end(),
                      [&](const WorkItem &a, const WorkItem &b) { return cost_of(a) > cost_of(b); });
-    std::vector<long long> cost;
-    for (const WorkItem &it : items) cost.push_back(cost_of(it));
+    std::vector<long long> cost, cost_two_heads;
+    for (const WorkItem &it : items) {
+        cost.push_back(cost_of(it));
+        // An item of one query tile leaves the CTA's other tile slot idle; run it for two heads at
+        // once instead (each slot with a K/V stream of its own): the price of a two-tile unit, plus
+        // the second stream's tile loads.
+        cost_two_heads.push_back(it.q_rows > BM ? 0 : (long long)it.kv_blocks * 21 + 40);
+    }
     cudaFree(p->d_work);
     cudaFree(p->d_units);
     cudaFree(p->d_cta_begin);
@@ -780,7 +922,8 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
 
     HB_CUDA(cudaMalloc(&p->d_work, sizeof(WorkItem) * items.size()));
     HB_CUDA(cudaMemcpy(p->d_work, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
-    int rc = upload_schedule(items, cost, p->batch * p->heads, p->sm_count, &p->d_units, &p->d_cta_begin, &p->n_cta);
+    int rc = upload_schedule(items, cost, p->batch * p->heads, p->sm_count, &p->d_units, &p->d_cta_begin, &p->n_cta,
+                             &cost_two_heads);
     if (rc != HILBERTA_OK) return rc;
     // slice of heads for the pipelined host-buffer path: the largest divisor of `heads` not above heads / HB_HOST_SLICES (rounded up)
     p->chunk_heads = p->heads;
@@ -791,7 +934,7 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
         }
     if (p->chunk_heads < p->heads) {
         rc = upload_schedule(items, cost, p->batch * p->chunk_heads, p->sm_count, &p->d_units_chunk, &p->d_cta_begin_chunk,
-                             &p->n_cta_chunk);
+                             &p->n_cta_chunk, &cost_two_heads);
         if (rc != HILBERTA_OK) return rc;
     }
     {

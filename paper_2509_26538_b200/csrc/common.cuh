@@ -50,10 +50,13 @@ struct WorkItem {
 };
 
 // A work item applied to one (batch, head).  Units are assigned to CTAs on the
-// host (longest-processing-time-first) and stored grouped by CTA.
+// host (longest-processing-time-first) and stored grouped by CTA.  bh2 >= 0 (forward kernel
+// only, items of one query tile): the same item for a second (batch, head), which takes the
+// CTA's other query-tile slot with a K/V stream of its own.
 struct WorkUnit {
     int item;
     int bh;
+    int bh2;
 };
 
 }  // namespace hilberta
@@ -133,8 +136,11 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
 std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, int block);
 // HILBERTA_OK iff the list is safe to hand to a kernel (ranges inside [0, S), rows covered exactly once)
 int check_work_items(const WorkItem *items, int n, int S, int item_rows, int block);
+// cost_two_heads: nullptr, or per item the cost of running it for TWO (batch, head) indices in one unit
+// (0: the item is not paired); such items are emitted as units of two consecutive indices.
 int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
-                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out);
+                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out,
+                    const std::vector<long long> *cost_two_heads = nullptr);
 int attn_bf16_prepare(hilberta_plan_t *p);
 // attn_bf16_pair_sm100.cu: the forward kernel on pairs of SMs (bf16, head dim 128, inputs in physical order)
 int attn_bf16_pair_prepare(hilberta_plan_t *p);

@@ -556,7 +556,7 @@ extern "C" int hilberta_plan_export(const hilberta_plan_t *p, int what, void *ho
             dsrc = p->d_status + 32;
             if (host_buf) HB_CUDA(cudaDeviceSynchronize());
             break;
-#ifdef HB_TIMING
+#if defined(HB_TIMING) || defined(HB_STAMPS)
         case 100: need = sizeof(int) * 4096; dsrc = p->d_status; break;  // role cycle counters and event trace
 #endif
         default: return HILBERTA_ERR_INVALID;

@@ -89,21 +89,35 @@ int check_work_items(const WorkItem *items, int n, int S, int item_rows, int blo
 // items must be sorted by descending cost.  On success *d_units holds items.size() * bh units
 // grouped by CTA and *d_cta_begin the n_cta + 1 offsets (both device memory, owned by the caller).
 int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
-                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out) {
-    const long long n_units = (long long)items.size() * bh;
-    if (n_units > (1ll << 30)) return HILBERTA_ERR_INVALID;
+                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out, const std::vector<long long> *cost_two_heads) {
+    if ((long long)items.size() * bh > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    // all units with their costs, longest first (items arrive sorted; paired units may cost more than
+    // the single units of an earlier item, hence the stable sort)
+    struct Costed {
+        WorkUnit unit;
+        long long cost;
+    };
+    std::vector<Costed> all;
+    all.reserve(items.size() * (size_t)bh);
+    for (int i = 0; i < (int)items.size(); ++i) {
+        const long long two = cost_two_heads ? (*cost_two_heads)[i] : 0;
+        int j = 0;
+        if (two > 0)
+            for (; j + 1 < bh; j += 2) all.push_back(Costed{WorkUnit{i, j, j + 1}, two});
+        for (; j < bh; ++j) all.push_back(Costed{WorkUnit{i, j, -1}, cost[i]});
+    }
+    std::stable_sort(all.begin(), all.end(), [](const Costed &a, const Costed &b) { return a.cost > b.cost; });
+    const long long n_units = (long long)all.size();
     const int n_cta = (int)std::min<long long>(n_units, sm_count);
     std::vector<std::vector<WorkUnit>> bins(n_cta);
     typedef std::pair<long long, int> Load;  // (load, cta)
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
     for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
-    for (int i = 0; i < (int)items.size(); ++i) {
-        for (int j = 0; j < bh; ++j) {
-            Load top = heap.top();
-            heap.pop();
-            bins[top.second].push_back(WorkUnit{i, j});
-            heap.push(Load(top.first + cost[i], top.second));
-        }
+    for (const Costed &cu : all) {
+        Load top = heap.top();
+        heap.pop();
+        bins[top.second].push_back(cu.unit);
+        heap.push(Load(top.first + cu.cost, top.second));
     }
     std::vector<WorkUnit> units;
     std::vector<int> cta_begin(n_cta + 1, 0);
