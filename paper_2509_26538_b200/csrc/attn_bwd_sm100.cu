@@ -126,6 +126,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
                 const __grid_constant__ CUtensorMap tmT1, const __grid_constant__ CUtensorMap tmT2,
                 const Params prm) {
     extern __shared__ uint8_t smem_raw[];
+#ifdef HB_STAMPS
+    if (threadIdx.x == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        prm.status[1024 + MODE * 1024 + 4 * blockIdx.x] = (int)(ns & 0x7fffffff);
+    }
+#endif
     constexpr uint32_t REG_A = 0, REG_B = 128, OUT_A = 256, OUT_B = 384;   // TMEM columns
     constexpr int NSLAB = HD / 64;
     constexpr uint32_t TILE_TX = BM * HD * 2;                              // bytes of one tile
@@ -518,6 +525,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmR1, const __grid_constant_
         __syncwarp();
         tmem_dealloc(tmem, TMEM_COLS);
     }
+#ifdef HB_STAMPS
+    if (threadIdx.x == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        prm.status[1024 + MODE * 1024 + 4 * blockIdx.x + 1] = (int)(ns & 0x7fffffff);
+    }
+#endif
 }
 
 // lse2[row] = lse[row] * log2 e, delta[row] = sum_d dO[row, d] * O[row, d]: HD / 8 lanes per row
@@ -597,15 +611,21 @@ int attn_bwd_prepare(hilberta_plan_t *p) {
     const int rc = upload_schedule(items, cost, bh, p->sm_count, &p->d_bwd_units, &p->d_bwd_cta_begin, &p->n_bwd_cta);
     if (rc != HILBERTA_OK) return rc;
     HB_CUDA(cudaMalloc(&p->d_delta, sizeof(float) * 2 * (size_t)bh * p->S));
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        const void *kernels[4] = {(const void *)attn_bwd_kernel<MODE_DQ, 128>, (const void *)attn_bwd_kernel<MODE_DKV, 128>,
-                                  (const void *)attn_bwd_kernel<MODE_DQ, 64>, (const void *)attn_bwd_kernel<MODE_DKV, 64>};
-        for (int i = 0; i < 4 && attr_err == cudaSuccess; ++i)
-            attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    });
-    HB_CUDA(attr_err);
+    {
+        // The shared-memory opt-in is an attribute of the kernel ON ONE DEVICE: set it once for every
+        // device a plan is bound on (a failure is reported, not remembered).
+        static std::mutex attr_mutex;
+        static bool attr_done[64] = {};
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if (p->device < 0 || p->device >= 64) return HILBERTA_ERR_INVALID;
+        if (!attr_done[p->device]) {
+            const void *kernels[4] = {(const void *)attn_bwd_kernel<MODE_DQ, 128>, (const void *)attn_bwd_kernel<MODE_DKV, 128>,
+                                      (const void *)attn_bwd_kernel<MODE_DQ, 64>, (const void *)attn_bwd_kernel<MODE_DKV, 64>};
+            for (int i = 0; i < 4; ++i)
+                HB_CUDA(cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+            attr_done[p->device] = true;
+        }
+    }
     return HILBERTA_OK;
 }
 
