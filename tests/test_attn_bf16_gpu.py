@@ -253,3 +253,39 @@ def test_peaky_row_whose_largest_weight_sits_on_a_rounding_tie():
     assert np.isfinite(g_).all()
     assert (np.abs(g_ - ref) <= 1e-2 * np.maximum(1.0, np.abs(ref))).all(), float(np.abs(g_ - ref).max())
     assert orc.rel_l2_err(g_, ref) <= TOL_REL_L2
+
+
+@pytest.mark.parametrize("B,heads", [(2, 3), (1, 5), (1, 2)])
+def test_one_tile_items_paired_over_heads(B, heads):
+    """Every work item here has ONE query tile (56 prefix rows; slid tiles of at most 128 rows), so the
+    kernel runs each item for two (batch, head) indices at once, one per query-tile slot with its own
+    K/V stream -- across the batch boundary for (2, 3), with one index left over for odd counts.  Output
+    and log-sum-exp against the oracle, every row of every head; the fused exit gather must write the
+    same bits at the original positions."""
+    H, tile, o, hs, nt = 32, 128, 64, 4, 40
+    S = nt + H * H
+    g = torch.Generator().manual_seed(31 + 7 * B + heads)
+    q, k, v = (torch.randn((B, heads, S, 128), generator=g).bfloat16() for _ in range(3))
+    ig, grp = orc.token_classes(H, H, tile, o, hs, nt)
+    ref_out, ref_lse = attn_c.attention_rows(q.float().numpy(), k.float().numpy(), v.float().numpy(), ig, grp,
+                                             return_lse=True)
+    plan = hb.Plan(H, H, tile, o, hs, nt)
+    try:
+        p2o = torch.from_numpy(plan.export(hb.EXPORT_PHYS2ORIG).astype(np.int64))
+        qp, kp, vp = (t[:, :, p2o].contiguous().cuda() for t in (q, k, v))
+        plan.bind_like(qp)
+        outp = torch.full_like(qp, float("nan"))
+        lse = torch.full((B, heads, S), float("nan"), device="cuda", dtype=torch.float32)
+        plan.forward_lse(qp, kp, vp, outp, lse)
+        out_orig = torch.full_like(qp, float("nan"))
+        plan.forward_unpermute(qp, kp, vp, out_orig)
+        assert plan.status() == 0
+        got = torch.empty_like(q)
+        got[:, :, p2o] = outp.cpu()
+        got_lse = torch.empty((B, heads, S), dtype=torch.float64)
+        got_lse[:, :, p2o] = lse.cpu().double()
+    finally:
+        plan.destroy()
+    check(got, ref_out)
+    assert torch.equal(out_orig.cpu().view(torch.int16), got.view(torch.int16))
+    assert np.max(np.abs(got_lse.numpy() - ref_lse)) <= 2e-3
