@@ -184,10 +184,12 @@ int hilberta_plan_bind(hilberta_plan_t *plan, int batch, int heads, int head_dim
  * softmax; prefix queries read every key).
  *
  *   q, k, v   device pointers, PHYSICAL token order, layout as bound; read only.
- *   out       device pointer, same layout, written; must not overlap q, k or v.
- *             The call rejects `out` EQUAL to an input (ERR_INVALID); buffers that overlap
- *             partly are not detected (with strided, interleaved layouts overlapping
- *             address ranges are legitimate) and give undefined results.
+ *   out       device pointer, same layout, written; must not share a byte with q, k or v
+ *             (ERR_INVALID otherwise).  The test is exact on the bound strides (see
+ *             hilberta_check_overlap), so q, k, v and out may be slices of one packed,
+ *             interleaved buffer as long as no element of out is an element of an input.
+ *             (e4m3 inputs and their bf16 output have different byte strides: there the
+ *             address ranges are compared, which also rejects interleaving.)
  *             bf16 and e4m3: all four 16-byte aligned.
  *   values    q, k and v must be finite over the WHOLE tensors: the tensor-core kernels
  *             multiply the rows of a partly masked 128-key block by weights that are
@@ -230,9 +232,9 @@ int hilberta_forward_lse(const void *q, const void *k, const void *v, void *out,
  * carries lse * log2(e) and delta between the launches, so two backward calls on
  * the same plan must not overlap on the device.
  *
- * Errors: ERR_INVALID (NULL or misaligned pointers, an output equal to another
- * argument, wrong device), ERR_UNBOUND, ERR_CUDA.  Partly overlapping buffers are
- * not detected (see hilberta_forward). */
+ * Errors: ERR_INVALID (NULL or misaligned pointers, an output that shares a byte with
+ * another tensor argument -- the exact test of hilberta_check_overlap --, wrong
+ * device), ERR_UNBOUND, ERR_CUDA. */
 int hilberta_backward(const void *dout, const void *q, const void *k, const void *v, const void *out,
                       const float *lse, void *dq, void *dk, void *dv, const hilberta_plan_t *plan,
                       void *stream);
@@ -340,6 +342,16 @@ int hilberta_plan_status(hilberta_plan_t *plan);
  * items' query ranges cover [0, S) exactly once.  Otherwise ERR_INVALID.  (Sec. 3.2 / 3.3: every
  * query row belongs to the prefix or to exactly one slid tile.) */
 int hilberta_check_work_list(const int32_t *items, int n_items, int S, int item_rows, int block);
+
+/* Host-side aliasing test the attention calls run on their pointer arguments (no GPU involved).
+ * Two tensors of the layout [batch, heads, S, row] with the same BYTE strides and rows of row_bytes
+ * contiguous bytes, at base addresses a and b: returns 1 if they share at least one byte, else 0.
+ * Exact (not a comparison of address ranges): they overlap iff b - a equals
+ * dx stride_b + dy stride_h + dz stride_s + dc for some |dx| < batch, |dy| < heads, |dz| < S,
+ * |dc| < row_bytes.  Algorithm 1 reads K and V blocks of other query blocks' launches in flight, so an
+ * output that aliases an input would race; interleaved slices of one buffer are fine. */
+int hilberta_check_overlap(uint64_t a, uint64_t b, int batch, int heads, int S, int64_t stride_b_bytes,
+                           int64_t stride_h_bytes, int64_t stride_s_bytes, int64_t row_bytes);
 
 /* Failure-detection self-test: launches a one-warp kernel that waits, with a 1 ms
  * deadline, on a barrier nothing arrives on -- the same bounded wait every role of

@@ -30,7 +30,7 @@ SYMBOLS = (
     "hilberta_backward_static", "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
-    "hilberta_check_work_list",
+    "hilberta_check_work_list", "hilberta_check_overlap",
     "hilberta_plan_status", "hilberta_selftest_timeout", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
     "hilberta_last_cuda_error",
 )
@@ -90,6 +90,9 @@ def lib():
         f.restype = i32
     L.hilberta_check_work_list.argtypes = [vp, i32, i32, i32, i32]
     L.hilberta_check_work_list.restype = i32
+    i64, u64 = ctypes.c_int64, ctypes.c_uint64
+    L.hilberta_check_overlap.argtypes = [u64, u64, i32, i32, i32, i64, i64, i64, i64]
+    L.hilberta_check_overlap.restype = i32
     L.hilberta_selftest_timeout.argtypes = [vp, vp]
     L.hilberta_selftest_timeout.restype = i32
     L.hilberta_plan_status.argtypes = [vp]
@@ -110,6 +113,13 @@ def check_work_list(items, S: int, item_rows: int, block: int) -> int:
     """Status of hilberta_check_work_list for an [n, 10] int32 array of work items (host only)."""
     a = np.ascontiguousarray(items, dtype=np.int32).reshape(-1, 10)
     return int(lib().hilberta_check_work_list(a.ctypes.data, a.shape[0], int(S), int(item_rows), int(block)))
+
+
+def check_overlap(a: int, b: int, batch: int, heads: int, S: int, stride_b: int, stride_h: int, stride_s: int,
+                  row_bytes: int) -> bool:
+    """hilberta_check_overlap: do two [batch, heads, S, row] tensors with these byte strides share a byte? (host only)"""
+    return bool(lib().hilberta_check_overlap(int(a), int(b), int(batch), int(heads), int(S), int(stride_b),
+                                             int(stride_h), int(stride_s), int(row_bytes)))
 
 
 def _check(status: int, where: str):

@@ -723,21 +723,22 @@ extern "C" int hilberta_backward_static(const void *dout, const void *q, const v
                                         const hilberta_plan_t *p, void *stream) {
     if (!p || !dout || !q || !k || !v || !out || !lse || !dq || !dk || !dv) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    const void *in[5] = {dout, q, k, v, out};
-    void *outs[3] = {dq, dk, dv};
-    uintptr_t bits = ((uintptr_t)lse & 3) ? 15 : 0;
-    for (int i = 0; i < 3; ++i) {
-        bits |= (uintptr_t)outs[i];
-        for (int j = 0; j < 5; ++j)
-            if (outs[i] == in[j]) return HILBERTA_ERR_INVALID;
-        for (int j = 0; j < i; ++j)
-            if (outs[i] == outs[j]) return HILBERTA_ERR_INVALID;
-    }
-    for (int j = 0; j < 5; ++j) bits |= (uintptr_t)in[j];
-    if (bits & 15) return HILBERTA_ERR_INVALID;
     // two floats of scratch per (batch, head, token): refuse what the fixed array cannot hold
     if (2ull * p->batch * p->heads * p->S > (unsigned long long)HILBERTA_STATIC_SCRATCH_FLOATS)
         return HILBERTA_ERR_BUFFER;
+    const void *in[5] = {dout, q, k, v, out};
+    void *outs[3] = {dq, dk, dv};
+    uintptr_t bits = ((uintptr_t)lse & 3) ? 15 : 0;
+    const size_t esz = p->dtype == HILBERTA_FP32 ? 4 : 2;
+    for (int i = 0; i < 3; ++i) {
+        bits |= (uintptr_t)outs[i];
+        for (int j = 0; j < 5; ++j)
+            if (hilberta::bound_tensors_overlap(p, outs[i], esz, in[j], esz)) return HILBERTA_ERR_INVALID;
+        for (int j = 0; j < i; ++j)
+            if (hilberta::bound_tensors_overlap(p, outs[i], esz, outs[j], esz)) return HILBERTA_ERR_INVALID;
+    }
+    for (int j = 0; j < 5; ++j) bits |= (uintptr_t)in[j];
+    if (bits & 15) return HILBERTA_ERR_INVALID;
     int dev = -1;
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;

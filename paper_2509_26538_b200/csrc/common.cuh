@@ -155,4 +155,6 @@ int launch_attn_fp32_bwd(const hilberta_plan_t *p, const void *dout, const void 
                          const void *out, const float *lse, void *dq, void *dk, void *dv, float *delta,
                          cudaStream_t stream);
 int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream);
+// plan.cu: does a written tensor share a byte with another tensor of the bound layout?
+bool bound_tensors_overlap(const hilberta_plan_t *p, const void *out, size_t esz_out, const void *in, size_t esz_in);
 }  // namespace hilberta

@@ -619,12 +619,66 @@ extern "C" int hilberta_plan_bind(hilberta_plan_t *p, int batch, int heads, int 
     return HILBERTA_OK;
 }
 
+// Do two tensors of the layout [batch, heads, S, row] share a byte?  Both use the byte strides sb, sh,
+// ss and rows of row_bytes contiguous bytes; a and b are their base addresses.  Exact: the tensors
+// overlap iff b - a = dx sb + dy sh + dz ss + dc for some |dx| < batch, |dy| < heads, |dz| < S,
+// |dc| < row_bytes (every such difference of indices is the difference of two valid indices).  So
+// tensors interleaved in one buffer (q, k, v and out as slices of one packed array) pass, and any
+// real overlap -- a shifted copy of an input used as output -- is caught.
+static bool layouts_overlap(uint64_t a, uint64_t b, int batch, int heads, int S, int64_t sb, int64_t sh, int64_t ss,
+                            int64_t row_bytes) {
+    if (batch < 1 || heads < 1 || S < 1 || row_bytes < 1) return false;
+    const int64_t d = (int64_t)(b - a);
+    if (ss <= 0) {
+        // no usable token stride: compare the address ranges
+        const int64_t ext = (batch - 1) * llabs(sb) + (heads - 1) * llabs(sh) + (int64_t)(S - 1) * llabs(ss) + row_bytes;
+        return d < ext && -d < ext;
+    }
+    for (int dx = -(batch - 1); dx <= batch - 1; ++dx)
+        for (int dy = -(heads - 1); dy <= heads - 1; ++dy) {
+            const int64_t rem = d - dx * sb - dy * sh;
+            int64_t dz = rem / ss;   // rem = dz ss + dc: dz is the quotient rounded toward zero or its neighbours
+            for (int64_t z = dz - 1; z <= dz + 1; ++z)
+                if (z > -(int64_t)S && z < (int64_t)S && llabs(rem - z * ss) < row_bytes) return true;
+        }
+    return false;
+}
+
+extern "C" int hilberta_check_overlap(uint64_t a, uint64_t b, int batch, int heads, int S, int64_t stride_b_bytes,
+                                      int64_t stride_h_bytes, int64_t stride_s_bytes, int64_t row_bytes) {
+    return layouts_overlap(a, b, batch, heads, S, stride_b_bytes, stride_h_bytes, stride_s_bytes, row_bytes) ? 1 : 0;
+}
+
+namespace hilberta {
+// `out` (element size esz_out) against `in` (element size esz_in) on the plan's bound layout.  Equal
+// element sizes: the exact test.  e4m3 inputs with a bf16 output use different byte strides: there
+// the address ranges are compared.
+bool bound_tensors_overlap(const hilberta_plan_t *p, const void *out, size_t esz_out, const void *in, size_t esz_in) {
+    const uint64_t a = (uint64_t)(uintptr_t)out, b = (uint64_t)(uintptr_t)in;
+    if (esz_out == esz_in)
+        return layouts_overlap(a, b, p->batch, p->heads, p->S, p->stride_b * (int64_t)esz_out, p->stride_h * (int64_t)esz_out,
+                               p->stride_s * (int64_t)esz_out, (int64_t)p->head_dim * (int64_t)esz_out);
+    auto extent = [&](size_t esz) {
+        return (uint64_t)(((int64_t)(p->batch - 1) * p->stride_b + (int64_t)(p->heads - 1) * p->stride_h +
+                           (int64_t)(p->S - 1) * p->stride_s + p->head_dim) * (int64_t)esz);
+    };
+    return a < b + extent(esz_in) && b < a + extent(esz_out);
+}
+}  // namespace hilberta
+
 static int forward_impl(const void *q, const void *k, const void *v, void *out, float *lse,
                         const hilberta_plan_t *p, const int *out_map, const int *in_map, void *stream,
                         int chunk = -1) {
     if (!p || !q || !k || !v || !out) return HILBERTA_ERR_INVALID;
     if (!p->bound) return HILBERTA_ERR_UNBOUND;
-    if (out == q || out == k || out == v) return HILBERTA_ERR_INVALID;
+    {
+        // `out` must not share a byte with an input (other launches' reads would race with its writes)
+        const size_t esz_in = p->dtype == HILBERTA_BF16 ? 2 : p->dtype == HILBERTA_FP8_E4M3 ? 1 : 4;
+        const size_t esz_out = p->dtype == HILBERTA_FP8_E4M3 ? 2 : esz_in;
+        const void *in[3] = {q, k, v};
+        for (int i = 0; i < 3; ++i)
+            if (hilberta::bound_tensors_overlap(p, out, esz_out, in[i], esz_in)) return HILBERTA_ERR_INVALID;
+    }
     int dev = -1;
     HB_CUDA(cudaGetDevice(&dev));
     if (dev != p->device) return HILBERTA_ERR_INVALID;  // the plan's tables live on another device
@@ -665,12 +719,13 @@ extern "C" int hilberta_backward(const void *dout, const void *q, const void *k,
     const void *in[5] = {dout, q, k, v, out};
     void *outs[3] = {dq, dk, dv};
     uintptr_t bits = (uintptr_t)lse & 3 ? 15 : 0;
+    const size_t esz = p->dtype == HILBERTA_FP32 ? 4 : 2;
     for (int i = 0; i < 3; ++i) {
         bits |= (uintptr_t)outs[i];
         for (int j = 0; j < 5; ++j)
-            if (outs[i] == in[j]) return HILBERTA_ERR_INVALID;
+            if (hilberta::bound_tensors_overlap(p, outs[i], esz, in[j], esz)) return HILBERTA_ERR_INVALID;
         for (int j = 0; j < i; ++j)
-            if (outs[i] == outs[j]) return HILBERTA_ERR_INVALID;
+            if (hilberta::bound_tensors_overlap(p, outs[i], esz, outs[j], esz)) return HILBERTA_ERR_INVALID;
     }
     for (int j = 0; j < 5; ++j) bits |= (uintptr_t)in[j];
     if (bits & 15) return HILBERTA_ERR_INVALID;

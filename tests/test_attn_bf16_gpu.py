@@ -289,3 +289,36 @@ def test_one_tile_items_paired_over_heads(B, heads):
     check(got, ref_out)
     assert torch.equal(out_orig.cpu().view(torch.int16), got.view(torch.int16))
     assert np.max(np.abs(got_lse.numpy() - ref_lse)) <= 2e-3
+
+
+def test_packed_buffer_is_accepted_and_aliasing_outputs_are_rejected():
+    """q, k, v and out as the four slices of ONE [B, S, 4, heads, D] buffer: their address ranges interleave
+    but no element is shared, so the call runs (and matches the oracle).  An output that shares bytes
+    with an input -- shifted by one head, by a few rows, or equal -- is refused before anything is launched."""
+    H, tile, o, hs, nt = 16, 64, 16, 2, 9
+    S, B, heads = nt + H * H, 2, 3
+    g = torch.Generator().manual_seed(6)
+    q, k, v = (torch.randn((B, heads, S, 128), generator=g).bfloat16() for _ in range(3))
+    ref = oracle_rows(H, tile, o, hs, nt, q, k, v)
+    plan = hb.Plan(H, H, tile, o, hs, nt)
+    try:
+        p2o = torch.from_numpy(plan.export(hb.EXPORT_PHYS2ORIG).astype(np.int64))
+        packed = torch.zeros((B, S, 4, heads, 128), dtype=torch.bfloat16, device="cuda")
+        views = [packed[:, :, i].permute(0, 2, 1, 3) for i in range(4)]   # [B, heads, S, D] views of the slices
+        for dst, src in zip(views, (q, k, v)):
+            dst.copy_(src[:, :, p2o].cuda())
+        qp, kp, vp, out = views
+        plan.bind_like(qp)
+        plan.forward(qp, kp, vp, out)
+        assert plan.status() == 0
+        got = torch.empty_like(q)
+        got[:, :, p2o] = out.cpu()
+        check(got, ref)
+        L = hb.lib()
+        launches = hb.launch_count()
+        one_head = 128 * 2
+        for bad in (qp.data_ptr(), kp.data_ptr() + one_head, vp.data_ptr() - one_head, qp.data_ptr() + 3 * packed.stride(1) * 2):
+            assert L.hilberta_forward(qp.data_ptr(), kp.data_ptr(), vp.data_ptr(), bad, plan._h, None) == hb.ERR_INVALID
+        assert hb.launch_count() == launches
+    finally:
+        plan.destroy()
