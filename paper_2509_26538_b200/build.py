@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhilberta.so")
-SOURCES = ["plan.cu", "schedule.cu", "permute.cu", "attn_fp32.cu", "attn_fp32_bwd.cu", "attn_bf16_sm100.cu", "attn_bf16_pair_sm100.cu", "attn_bwd_sm100.cu"]
+SOURCES = ["plan.cu", "schedule.cu", "permute.cu", "attn_fp32.cu", "attn_fp32_bwd.cu", "attn_bf16_sm100.cu", "attn_bf16_pair_sm100.cu", "attn_bf16_solo_sm100.cu", "attn_bwd_sm100.cu"]
 HEADERS = ["common.cuh", "sm100_ptx.cuh", "attn_softmax_math.cuh"]
 
 

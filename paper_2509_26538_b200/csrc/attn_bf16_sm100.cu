@@ -954,6 +954,10 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
             attr_done[p->device] = true;
         }
     }
+    {
+        const int rc_solo = attn_bf16_solo_prepare(p);
+        if (rc_solo != HILBERTA_OK) return rc_solo;
+    }
     return attn_bf16_pair_prepare(p);
 }
 
@@ -961,14 +965,21 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
                      float *lse, const int *out_map, const int *in_map, cudaStream_t stream, int chunk) {
     if (p->n_work == 0) return HILBERTA_OK;
     // bf16 with head dim 128 and inputs in physical order can also run on pairs of SMs
-    // (attn_bf16_pair_sm100.cu).  That kernel is correct but measures slower than this one, so it is
-    // opt-in: the environment variable HILBERTA_FORWARD_KERNEL=pair selects it (read once).
+    // (attn_bf16_pair_sm100.cu) or with one query tile per CTA (attn_bf16_solo_sm100.cu).  Those kernels
+    // are correct but measure slower than this one, so they are opt-in: the environment variable
+    // HILBERTA_FORWARD_KERNEL=pair or =solo selects them (read once).
     static const bool use_pair = [] {
         const char *e = getenv("HILBERTA_FORWARD_KERNEL");
         return e && e[0] == 'p';
     }();
     if (use_pair && !in_map && chunk < 0 && p->n_pair > 0)
         return launch_attn_bf16_pair(p, q, k, v, out, lse, out_map, stream);
+    static const bool use_solo = [] {
+        const char *e = getenv("HILBERTA_FORWARD_KERNEL");
+        return e && e[0] == 's';
+    }();
+    if (use_solo && !in_map && chunk < 0 && p->n_solo > 0)
+        return launch_attn_bf16_solo(p, q, k, v, out, lse, out_map, stream);
     int heads = p->heads, n_cta = p->n_cta;
     const WorkUnit *units = p->d_units;
     const int *cta_begin = p->d_cta_begin;

@@ -101,6 +101,11 @@ struct hilberta_plan_s {
     hilberta::WorkUnit *d_units_pair;
     int *d_pair_begin;
     int n_pair;
+    // the one-tile kernel's work list and schedule (bf16, head dim 128): items of 128 rows
+    hilberta::WorkItem *d_work_solo;
+    hilberta::WorkUnit *d_units_solo;
+    int *d_solo_begin;
+    int n_solo;
     cudaStream_t s_in, s_out;           // copy streams of hilberta_forward_host (created on first use)
     std::vector<cudaEvent_t> ev_in, ev_done;
     // backward pass: 128-row items over the same key lists, their schedule, and the
@@ -145,6 +150,11 @@ int attn_bf16_prepare(hilberta_plan_t *p);
 // attn_bf16_pair_sm100.cu: the forward kernel on pairs of SMs (bf16, head dim 128, inputs in physical order)
 int attn_bf16_pair_prepare(hilberta_plan_t *p);
 int launch_attn_bf16_pair(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
+                          float *lse, const int *out_map, cudaStream_t stream);
+// attn_bf16_solo_sm100.cu: the forward kernel with one query tile per CTA and double-buffered scores
+// (bf16, head dim 128, inputs in physical order)
+int attn_bf16_solo_prepare(hilberta_plan_t *p);
+int launch_attn_bf16_solo(const hilberta_plan_t *p, const void *q, const void *k, const void *v, void *out,
                           float *lse, const int *out_map, cudaStream_t stream);
 int attn_bwd_prepare(hilberta_plan_t *p);
 // dq, dk, dv (bf16, physical order, the bound strides) from dout, q, k, v, out and the forward's lse.

@@ -289,6 +289,9 @@ static void free_plan(hilberta_plan_t *p) {
     cudaFree(p->d_work_pair);
     cudaFree(p->d_units_pair);
     cudaFree(p->d_pair_begin);
+    cudaFree(p->d_work_solo);
+    cudaFree(p->d_units_solo);
+    cudaFree(p->d_solo_begin);
     cudaFree(p->d_cta_begin_chunk);
     for (cudaEvent_t e : p->ev_in) cudaEventDestroy(e);
     for (cudaEvent_t e : p->ev_done) cudaEventDestroy(e);

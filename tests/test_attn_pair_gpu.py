@@ -1,9 +1,10 @@
-"""The forward kernel on pairs of SMs (two-CTA tensor-core mode) against the fp64 oracle.
+"""The two alternative forward kernels against the fp64 oracle: `pair` (pairs of SMs, two-CTA
+tensor-core mode) and `solo` (one query tile per CTA with double-buffered scores).
 
-The pair kernel is opt-in through the environment variable HILBERTA_FORWARD_KERNEL=pair, which the
-library reads once per process.  So this test runs the bf16 forward and log-sum-exp parity tests
-again in a child process with that variable set: the same cases, the same tolerances (max-abs
-<= 1e-2, relative L2 <= 5e-3, same launch twice bit-identical), the other kernel."""
+Both are opt-in through the environment variable HILBERTA_FORWARD_KERNEL, which the library reads
+once per process.  So this test runs the bf16 forward and log-sum-exp parity tests again in a child
+process with that variable set: the same cases, the same tolerances (max-abs <= 1e-2, relative L2
+<= 5e-3, same launch twice bit-identical), the other kernel."""
 import os
 import subprocess
 import sys
@@ -15,8 +16,9 @@ pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def test_pair_kernel_passes_the_bf16_parity_tests():
-    env = dict(os.environ, HILBERTA_FORWARD_KERNEL="pair")
+@pytest.mark.parametrize("kernel", ["pair", "solo"])
+def test_alternative_kernel_passes_the_bf16_parity_tests(kernel):
+    env = dict(os.environ, HILBERTA_FORWARD_KERNEL=kernel)
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
            os.path.join(ROOT, "tests", "test_attn_bf16_gpu.py"), os.path.join(ROOT, "tests", "test_lse_gpu.py"),
            "-k", "not largest_grid and not flux4096"]
