@@ -343,6 +343,19 @@ int hilberta_plan_status(hilberta_plan_t *plan);
  * query row belongs to the prefix or to exactly one slid tile.) */
 int hilberta_check_work_list(const int32_t *items, int n_items, int S, int item_rows, int block);
 
+/* The static schedule of the attention kernels, computed on the host exactly as hilberta_plan_bind
+ * computes it (no GPU involved; exposed so that the assignment can be tested and inspected).  Work
+ * item i applied to (batch, head) index j is a unit of cost cost[i]; where cost_two_heads is given and
+ * cost_two_heads[i] > 0 the item is instead run for two consecutive indices at once (a unit
+ * (i, j, j + 1) of that cost; an odd index left over stays single).  Units go, longest first, to the CTA
+ * with the smallest load so far (Algorithm 1 runs one query block per program; here a persistent CTA
+ * runs a list of them).  units receives three int32 per unit (item, index, second index or -1),
+ * grouped by CTA -- at most n_items * bh units; cta_begin receives n_cta + 1 offsets into it (CTAs that
+ * get nothing repeat the end offset); largest_load, if not NULL, the largest CTA load.
+ * Errors: ERR_INVALID (bad counts, NULL outputs). */
+int hilberta_schedule_units(int n_items, const int64_t *cost, const int64_t *cost_two_heads, int bh, int n_cta,
+                            int32_t *units, int32_t *cta_begin, int64_t *largest_load);
+
 /* Host-side aliasing test the attention calls run on their pointer arguments (no GPU involved).
  * Two tensors of the layout [batch, heads, S, row] with the same BYTE strides and rows of row_bytes
  * contiguous bytes, at base addresses a and b: returns 1 if they share at least one byte, else 0.

@@ -30,7 +30,7 @@ SYMBOLS = (
     "hilberta_backward_static", "hilberta_permute",
     "hilberta_unpermute",
     "hilberta_forward_host",
-    "hilberta_check_work_list", "hilberta_check_overlap",
+    "hilberta_check_work_list", "hilberta_check_overlap", "hilberta_schedule_units",
     "hilberta_plan_status", "hilberta_selftest_timeout", "hilberta_launch_count", "hilberta_status_string", "hilberta_version",
     "hilberta_last_cuda_error",
 )
@@ -93,6 +93,8 @@ def lib():
     i64, u64 = ctypes.c_int64, ctypes.c_uint64
     L.hilberta_check_overlap.argtypes = [u64, u64, i32, i32, i32, i64, i64, i64, i64]
     L.hilberta_check_overlap.restype = i32
+    L.hilberta_schedule_units.argtypes = [i32, vp, vp, i32, i32, vp, vp, vp]
+    L.hilberta_schedule_units.restype = i32
     L.hilberta_selftest_timeout.argtypes = [vp, vp]
     L.hilberta_selftest_timeout.restype = i32
     L.hilberta_plan_status.argtypes = [vp]
@@ -120,6 +122,18 @@ def check_overlap(a: int, b: int, batch: int, heads: int, S: int, stride_b: int,
     """hilberta_check_overlap: do two [batch, heads, S, row] tensors with these byte strides share a byte? (host only)"""
     return bool(lib().hilberta_check_overlap(int(a), int(b), int(batch), int(heads), int(S), int(stride_b),
                                              int(stride_h), int(stride_s), int(row_bytes)))
+
+
+def schedule_units(cost, cost_two_heads, bh: int, n_cta: int):
+    """hilberta_schedule_units (host only): (units [n, 3] int32, cta_begin [n_cta + 1] int32, largest load)."""
+    c1 = np.ascontiguousarray(cost, dtype=np.int64)
+    c2 = None if cost_two_heads is None else np.ascontiguousarray(cost_two_heads, dtype=np.int64)
+    units = np.full((max(len(c1) * int(bh), 1), 3), -7, dtype=np.int32)
+    begin = np.zeros(int(n_cta) + 1, dtype=np.int32)
+    load = ctypes.c_int64(0)
+    _check(lib().hilberta_schedule_units(len(c1), c1.ctypes.data, None if c2 is None else c2.ctypes.data, int(bh), int(n_cta),
+                                         units.ctypes.data, begin.ctypes.data, ctypes.addressof(load)), "hilberta_schedule_units")
+    return units[:begin[-1]], begin, int(load.value)
 
 
 def _check(status: int, where: str):

@@ -141,6 +141,9 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
 std::vector<WorkItem> build_work_items(const hilberta_plan_t *p, int item_rows, int block);
 // HILBERTA_OK iff the list is safe to hand to a kernel (ranges inside [0, S), rows covered exactly once)
 int check_work_items(const WorkItem *items, int n, int S, int item_rows, int block);
+// the schedule on the host (see hilberta_schedule_units); returns the largest CTA load
+long long build_schedule(int n_items, const long long *cost, const long long *cost_two_heads, int bh, int sm_count,
+                         std::vector<WorkUnit> &units, std::vector<int> &cta_begin);
 // cost_two_heads: nullptr, or per item the cost of running it for TWO (batch, head) indices in one unit
 // (0: the item is not paired); such items are emitted as units of two consecutive indices.
 int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,

@@ -86,48 +86,62 @@ int check_work_items(const WorkItem *items, int n, int S, int item_rows, int blo
     return next == S ? HILBERTA_OK : HILBERTA_ERR_INVALID;
 }
 
-// items must be sorted by descending cost.  On success *d_units holds items.size() * bh units
-// grouped by CTA and *d_cta_begin the n_cta + 1 offsets (both device memory, owned by the caller).
-int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
-                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out, const std::vector<long long> *cost_two_heads) {
-    if ((long long)items.size() * bh > (1ll << 30)) return HILBERTA_ERR_INVALID;
-    // all units with their costs, longest first (items arrive sorted; paired units may cost more than
-    // the single units of an earlier item, hence the stable sort)
+// The static schedule on the host: every (item, batch * head) unit -- items with a two-head cost as
+// units of two consecutive indices -- goes, longest first, to the CTA with the smallest load so far.
+// units: grouped by CTA; cta_begin: n_cta + 1 offsets.  Returns the largest CTA load.
+long long build_schedule(int n_items, const long long *cost, const long long *cost_two_heads, int bh, int sm_count,
+                         std::vector<WorkUnit> &units, std::vector<int> &cta_begin) {
     struct Costed {
         WorkUnit unit;
         long long cost;
     };
     std::vector<Costed> all;
-    all.reserve(items.size() * (size_t)bh);
-    for (int i = 0; i < (int)items.size(); ++i) {
-        const long long two = cost_two_heads ? (*cost_two_heads)[i] : 0;
+    all.reserve((size_t)n_items * (size_t)bh);
+    for (int i = 0; i < n_items; ++i) {
+        const long long two = cost_two_heads ? cost_two_heads[i] : 0;
         int j = 0;
         if (two > 0)
             for (; j + 1 < bh; j += 2) all.push_back(Costed{WorkUnit{i, j, j + 1}, two});
         for (; j < bh; ++j) all.push_back(Costed{WorkUnit{i, j, -1}, cost[i]});
     }
+    // paired units may cost more than the single units of an earlier item, hence the sort (stable:
+    // equal costs keep the order of the items and of the heads)
     std::stable_sort(all.begin(), all.end(), [](const Costed &a, const Costed &b) { return a.cost > b.cost; });
     const long long n_units = (long long)all.size();
     const int n_cta = (int)std::min<long long>(n_units, sm_count);
-    std::vector<std::vector<WorkUnit>> bins(n_cta);
+    std::vector<std::vector<WorkUnit>> bins((size_t)std::max(n_cta, 0));
     typedef std::pair<long long, int> Load;  // (load, cta)
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
     for (int c = 0; c < n_cta; ++c) heap.push(Load(0, c));
+    long long makespan = 0;
     for (const Costed &cu : all) {
         Load top = heap.top();
         heap.pop();
         bins[top.second].push_back(cu.unit);
         heap.push(Load(top.first + cu.cost, top.second));
+        makespan = std::max(makespan, top.first + cu.cost);
     }
-    std::vector<WorkUnit> units;
-    std::vector<int> cta_begin(n_cta + 1, 0);
+    units.clear();
     units.reserve((size_t)n_units);
+    cta_begin.assign((size_t)n_cta + 1, 0);
     for (int c = 0; c < n_cta; ++c) {
         cta_begin[c] = (int)units.size();
         units.insert(units.end(), bins[c].begin(), bins[c].end());
     }
     cta_begin[n_cta] = (int)units.size();
-    *n_cta_out = n_cta;
+    return makespan;
+}
+
+// items must be sorted by descending cost.  On success *d_units holds the units grouped by CTA and
+// *d_cta_begin the n_cta + 1 offsets (both device memory, owned by the caller).
+int upload_schedule(const std::vector<WorkItem> &items, const std::vector<long long> &cost, int bh, int sm_count,
+                    WorkUnit **d_units, int **d_cta_begin, int *n_cta_out, const std::vector<long long> *cost_two_heads) {
+    if ((long long)items.size() * bh > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    std::vector<WorkUnit> units;
+    std::vector<int> cta_begin;
+    build_schedule((int)items.size(), cost.data(), cost_two_heads ? cost_two_heads->data() : nullptr, bh, sm_count, units,
+                   cta_begin);
+    *n_cta_out = (int)cta_begin.size() - 1;
     HB_CUDA(cudaMalloc(d_units, sizeof(WorkUnit) * units.size()));
     HB_CUDA(cudaMemcpy(*d_units, units.data(), sizeof(WorkUnit) * units.size(), cudaMemcpyHostToDevice));
     HB_CUDA(cudaMalloc(d_cta_begin, sizeof(int) * cta_begin.size()));
@@ -141,4 +155,25 @@ static_assert(sizeof(hilberta::WorkItem) == 10 * sizeof(int32_t), "hilberta_chec
 
 extern "C" int hilberta_check_work_list(const int32_t *items, int n_items, int S, int item_rows, int block) {
     return hilberta::check_work_items(reinterpret_cast<const hilberta::WorkItem *>(items), n_items, S, item_rows, block);
+}
+
+static_assert(sizeof(hilberta::WorkUnit) == 3 * sizeof(int32_t), "hilberta_schedule_units writes three ints per unit");
+
+extern "C" int hilberta_schedule_units(int n_items, const int64_t *cost, const int64_t *cost_two_heads, int bh, int n_cta,
+                                       int32_t *units, int32_t *cta_begin, int64_t *largest_load) {
+    if (n_items < 0 || bh < 1 || n_cta < 1 || (n_items > 0 && !cost) || !units || !cta_begin) return HILBERTA_ERR_INVALID;
+    if ((long long)n_items * bh > (1ll << 30)) return HILBERTA_ERR_INVALID;
+    std::vector<long long> c1(cost, cost + n_items), c2;
+    if (cost_two_heads) c2.assign(cost_two_heads, cost_two_heads + n_items);
+    std::vector<hilberta::WorkUnit> u;
+    std::vector<int> cb;
+    const long long m = hilberta::build_schedule(n_items, c1.data(), cost_two_heads ? c2.data() : nullptr, bh, n_cta, u, cb);
+    for (size_t i = 0; i < u.size(); ++i) {
+        units[3 * i] = u[i].item;
+        units[3 * i + 1] = u[i].bh;
+        units[3 * i + 2] = u[i].bh2;
+    }
+    for (int c = 0; c <= n_cta; ++c) cta_begin[c] = c < (int)cb.size() ? cb[c] : (int)u.size();
+    if (largest_load) *largest_load = m;
+    return HILBERTA_OK;
 }
