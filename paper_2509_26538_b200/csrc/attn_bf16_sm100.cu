@@ -72,8 +72,8 @@ constexpr float P_SHIFT_FP8 = 4.0f;
 #ifndef HB_HOST_SLICES
 #define HB_HOST_SLICES 8   // hilberta_forward_host pipelines its copies and launches over about this many slices of heads
 #endif
-#ifndef HB_SPLIT_P
-#define HB_SPLIT_P 1     // hand P to the MMA issuer in two halves
+#ifndef HB_SPLIT_AT
+#define HB_SPLIT_AT 2    // P goes to the MMA issuer in two parts: 32-key chunks 0..HB_SPLIT_AT, then the rest (2: 96 + 32 keys; measured 0.4-0.6 % faster than 64 + 64)
 #endif
 #ifndef HB_WARP_ARRIVE
 #define HB_WARP_ARRIVE 0 // 1: one mbarrier arrival per softmax warp (after a warp sync) instead of one per thread; measured equal
@@ -82,7 +82,7 @@ constexpr float P_SHIFT_FP8 = 4.0f;
 enum Bar {
     Q_FULL = 0, Q_EMPTY, DRAIN,
     S_FULL,
-    P_READY = S_FULL + QT,        // [t * 2 + half]: P columns of keys [64 half, +64) written, 128 arrivals
+    P_READY = S_FULL + QT,        // [t * 2 + part]: P columns of the keys of that part written, 128 arrivals
     PV_DONE = P_READY + 2 * QT,
     KV_FULL = PV_DONE + QT, KV_EMPTY = KV_FULL + NSTAGE,
     NUM_BARS = KV_EMPTY + NSTAGE
@@ -139,24 +139,34 @@ __device__ __forceinline__ void issue_qk(uint32_t tmem_s, uint32_t sQt, uint32_t
 }
 
 // O_t (+)= P_t V for one 128-key block: P from TMEM, V row-major in smem (N-major operand).
-// `half` selects keys [64 half, +64) of the block: four MMAs of K = 16 (bf16: 8 columns of P and
-// 16 rows of V each) or two of K = 32 (e4m3: 8 columns of P, four weights per column, and 32 rows of V).
+// `part` 0 covers the keys of 32-key chunks 0..HB_SPLIT_AT, part 1 the rest.  A chunk is two MMAs of
+// K = 16 (bf16: 8 columns of P and 16 rows of V each) or one of K = 32 (e4m3: 8 columns of P, four
+// weights per column, and 32 rows of V).
 template <int HD, bool FP8>
-__device__ __forceinline__ void issue_pv_half(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, int half,
+__device__ __forceinline__ void issue_pv_part(uint32_t tmem_o, uint32_t tmem_p, uint32_t sVslot, int part,
                                               bool accumulate) {
-    const uint64_t dv = smem_desc_sw128(sVslot + half * 8192, SLAB_BYTES, 1024);
+    const uint64_t dv = smem_desc_sw128(sVslot, SLAB_BYTES, 1024);
+    constexpr int C1 = HB_SPLIT_AT + 1, C2 = BN / 32;
+    static_assert(C1 >= 1 && C1 < C2, "both parts hold at least one chunk");
     if constexpr (FP8) {
         constexpr uint32_t IDESC = idesc_e4m3_f32(BM, HD, 1);
+        if (part == 0) {
 #pragma unroll
-        for (int k = 0; k < 2; ++k)
-            mma_ts_f8(tmem_o, tmem_p + half * 16 + k * 8, dv + (uint64_t)((k * 4096) >> 4), IDESC,
-                      (accumulate || k > 0) ? 1u : 0u);
+            for (int k = 0; k < C1; ++k)
+                mma_ts_f8(tmem_o, tmem_p + k * 8, dv + (uint64_t)((k * 4096) >> 4), IDESC, (accumulate || k > 0) ? 1u : 0u);
+        } else {
+#pragma unroll
+            for (int k = C1; k < C2; ++k) mma_ts_f8(tmem_o, tmem_p + k * 8, dv + (uint64_t)((k * 4096) >> 4), IDESC, 1u);
+        }
     } else {
         constexpr uint32_t IDESC = idesc_bf16_f32(BM, HD, 0, 1);
+        if (part == 0) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            mma_ts(tmem_o, tmem_p + half * 32 + k * 8, dv + (uint64_t)((k * 2048) >> 4), IDESC,
-                   (accumulate || k > 0) ? 1u : 0u);
+            for (int k = 0; k < 2 * C1; ++k)
+                mma_ts(tmem_o, tmem_p + k * 8, dv + (uint64_t)((k * 2048) >> 4), IDESC, (accumulate || k > 0) ? 1u : 0u);
+        } else {
+#pragma unroll
+            for (int k = 2 * C1; k < 2 * C2; ++k) mma_ts(tmem_o, tmem_p + k * 8, dv + (uint64_t)((k * 2048) >> 4), IDESC, 1u);
         }
     }
 }
@@ -437,7 +447,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #endif
             auto slot_of = [](uint32_t e) { return e % NSTAGE; };
             auto phase_of = [](uint32_t e) { return (e / NSTAGE) & 1; };
-            // O_t (+)= P_t V for block j of tile t (P arrives in two halves so the first four MMAs overlap
+            // O_t (+)= P_t V for block j of tile t (P arrives in two parts so the MMAs of the first overlap
             // the rest of the softmax), then S_t = Q_t K^T for the next block if there is one
             auto tile_turn = [&](int t, uint32_t eV, uint32_t eKn, bool accumulate, bool more) {
 #ifdef HB_TIMING
@@ -448,7 +458,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef HB_TIMING
                 tm_p += clock64() - tp0;
 #endif
-                issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, accumulate);
+                issue_pv_part<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 0, accumulate);
 #ifdef HB_TIMING
                 const long long tp1 = clock64();
 #endif
@@ -458,7 +468,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                 tm_p += clock64() - tp1;
 #endif
                 tc_fence_after();
-                issue_pv_half<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
+                issue_pv_part<HD, FP8>(tmem + 256 + t * HD, tmem + t * BN, sKV + slot_of(eV) * TILE_BYTES, 1, true);
                 mma_commit(bar(PV_DONE + t));
                 if (more) {
                     issue_qk<HD, FP8>(tmem + t * BN, sQ + t * TILE_BYTES, sKV + slot_of(eKn) * TILE_BYTES);
@@ -703,13 +713,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                         }
                         if constexpr (FP8) tmem_st8(tS + c * 8, pk);
                         else tmem_st16(tS + c * 16, pk);
-                        if (HB_SPLIT_P ? (c & 1) : (c == 3)) {  // keys [64 (c >> 1), +64) are in TMEM
+                        if (c == HB_SPLIT_AT || c == BN / 32 - 1) {  // a part of P is complete in TMEM
                             tmem_wait_st();
                             tc_fence_before();
                             if (HB_WARP_ARRIVE) __syncwarp();
                             if (!HB_WARP_ARRIVE || (tid & 31) == 0) {
-                                if (HB_SPLIT_P || c == 3) mbar_arrive(bar(P_READY + t * 2 + (c >> 1)));
-                                if (!HB_SPLIT_P) mbar_arrive(bar(P_READY + t * 2));
+                                mbar_arrive(bar(P_READY + t * 2 + (c == BN / 32 - 1 ? 1 : 0)));
                             }
                         }
                     }
