@@ -49,13 +49,21 @@ constexpr int BM = 128;        // rows per query tile
 constexpr int BN = 128;        // keys per block
 constexpr int QT = 2;          // query tiles per work item
 constexpr int ITEM_ROWS = QT * BM;
-constexpr int NSTAGE = 5;      // K/V ring slots (K0 V0 K1 V1 ...)
+constexpr int NSTAGE = 5;      // K/V ring slots at most (K0 V0 K1 V1 ...)
+// Ring slots of an instantiation.  The TMA kernels stage their output rows in shared memory (32 KB:
+// 4 KB per softmax warp) and store them with bulk tensor copies; with bf16 tiles of head dim 128 that
+// space is the fifth ring slot, which this kernel does not miss (measured equal with four), while the
+// gathering kernel does (40 % slower with four) and keeps five slots and per-lane stores.
+__host__ __device__ constexpr int ring_slots(bool gather, int hd, bool fp8) { return (!gather && !fp8 && hd == 128) ? 4 : NSTAGE; }
+constexpr int STAGE_BYTES = 8 * 4096;
 constexpr int SLAB_BYTES = BN * 128;     // one 64-column slab of 128 rows (128-byte swizzled rows)
 // bf16, head dim HD = 128: a tile is two slabs (32 KB); HD = 64: one slab (16 KB).
 // e4m3 (fp8 = true), HD = 128: rows of 128 bytes, one slab.
 __host__ __device__ constexpr int tile_bytes(int hd, bool fp8 = false) { return BN * hd * (fp8 ? 1 : 2); }
 constexpr int THREADS = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle (register donors)
-__host__ __device__ constexpr int smem_bytes(int hd, bool fp8 = false) { return (QT + NSTAGE) * tile_bytes(hd, fp8) + 1024; }
+__host__ __device__ constexpr int smem_bytes(int hd, bool fp8 = false, bool gather = false) {
+    return (QT + ring_slots(gather, hd, fp8)) * tile_bytes(hd, fp8) + (gather ? 0 : STAGE_BYTES) + 1024;
+}
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float RESCALE_THRESHOLD = 8.0f;        // log2 units
 // e4m3 weights: the running maximum may lag by 2^4 and every weight carries a factor 2^4 (divided
@@ -185,7 +193,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int sr
 template <bool GATHER, int HD, bool FP8 = false>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const KernelParams<GATHER> prm) {
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                 const KernelParams<GATHER> prm) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[NUM_BARS];
     __shared__ uint32_t tmem_slot;
@@ -200,6 +209,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
 #endif
     constexpr int TILE_BYTES = tile_bytes(HD, FP8);
+    constexpr int NS = ring_slots(GATHER, HD, FP8);
     constexpr int NSLAB = TILE_BYTES / SLAB_BYTES;
     using elem_t = typename std::conditional<FP8, uint8_t, __nv_bfloat16>::type;
     constexpr int EPC = 16 / (int)sizeof(elem_t);   // elements per 16-byte chunk
@@ -207,6 +217,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sQ = smem_u32(smem);
     const uint32_t sKV = sQ + QT * TILE_BYTES;
+    const uint32_t sStage = sKV + NS * TILE_BYTES;   // TMA kernels only: 4 KB per softmax warp
     const int tid = threadIdx.x, warp = tid >> 5;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -376,7 +387,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             bool ok = true;
             // one ring entry: the K or V tile at key row `row` of head (h, b)
             auto emit = [&](const CUtensorMap *tm, int row, int h, int b) {
-                const uint32_t s = kvc % NSTAGE, ph = (kvc / NSTAGE) & 1;
+                const uint32_t s = kvc % NS, ph = (kvc / NS) & 1;
                 ++kvc;
                 if (!wait_or_abort(bar(KV_EMPTY + s), ph ^ 1, &abort_flag, prm.status, 0x102)) return false;
                 mbar_expect_tx(bar(KV_FULL + s), TILE_BYTES);
@@ -445,8 +456,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #ifdef HB_TIMING
             long long tm_p = 0, tm_kv = 0, tm_start = clock64();
 #endif
-            auto slot_of = [](uint32_t e) { return e % NSTAGE; };
-            auto phase_of = [](uint32_t e) { return (e / NSTAGE) & 1; };
+            auto slot_of = [](uint32_t e) { return e % NS; };
+            auto phase_of = [](uint32_t e) { return (e / NS) & 1; };
             // O_t (+)= P_t V for block j of tile t (P arrives in two parts so the MMAs of the first overlap
             // the rest of the softmax), then S_t = Q_t K^T for the next block if there is one
             auto tile_turn = [&](int t, uint32_t eV, uint32_t eKn, bool accumulate, bool more) {
@@ -749,6 +760,42 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (prm.lse && row < wi.q_rows)
                 prm.lse[(long long)bh * prm.S + out_row] =
                     0.6931471805599453f * (m_ref - (FP8 ? P_SHIFT_FP8 : 0.f) + log2f(l));
+            // Rows through shared memory and one bulk tensor store per 64 columns and warp: the
+            // per-lane stores below cost 6 % of the launch at 2048^2 (10 % with 16 tiles at 1024^2)
+            // on the SM's load/store path.  Only where the output keeps the physical order and all
+            // 32 rows of the warp belong to the item (a box store would write the others too).
+            const int row0 = (dual ? 0 : t * BM) + (warp & 3) * 32;   // the warp's first row in the item
+            const bool bulk_out = !GATHER && (prm.out_align32 & 2) && row0 + 32 <= wi.q_rows;
+            if (bulk_out) {
+                const int lane = tid & 31;
+                const uint32_t slot = sStage + warp * 4096;
+#pragma unroll
+                for (int rd = 0; rd < HD / 64; ++rd) {
+                    // the bulk store that last used the slot has read it
+                    if (lane == 0) bulk_wait_group_read0();
+                    __syncwarp();
+#pragma unroll
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + rd * 64 + c2 * 32, o);
+                        tmem_wait_ld();
+                        uint32_t w[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            w[i] = pack_bf16(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
+                        // row `lane` of a 128-byte-swizzled box: 16-byte chunk k sits at k ^ (row & 7)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            st_shared_v4(slot + lane * 128 + (((c2 * 4 + k) ^ (lane & 7)) << 4), w + 4 * k);
+                    }
+                    fence_proxy_async_smem();   // generic-proxy writes -> the bulk copy's reads
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_4d(&tmO, slot, 64 * rd, wi.q_start + row0, h, b);
+                        bulk_commit_group();
+                    }
+                }
+            } else
 #pragma unroll
             for (int c = 0; c < HD / 32; ++c) {
                 uint32_t o[32];
@@ -759,7 +806,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
                         w[i] = pack_bf16(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
-                    if (prm.out_align32) {
+                    if (prm.out_align32 & 1) {
                         // 32-byte stores fill whole sectors: half the store instructions and
                         // half the L1/L2 write requests of 16-byte stores
 #pragma unroll
@@ -800,6 +847,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #endif
     }
 
+    // the epilogue's bulk stores are complete before the CTA gives up its shared memory
+    if (!GATHER && warp < 8 && (tid & 31) == 0) bulk_wait_group0();
     tc_fence_before();
     __syncthreads();
     if (blockIdx.x == 0 && tid == 0) {
@@ -883,6 +932,22 @@ int make_tensor_map(CUtensorMap *m, const void *base, const hilberta_plan_t *p, 
 
 namespace {
 
+// The output (always bf16) as a 4-D map with boxes of 64 columns x 32 rows, for the bulk stores of the
+// epilogue.  false: the layout does not qualify (base or a stride not a multiple of 16 bytes) and the
+// kernel keeps its per-lane stores.
+bool make_out_tensor_map(CUtensorMap *m, const void *out, const hilberta_plan_t *p, int heads) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    if (((uintptr_t)out & 15) != 0 || ((p->stride_b | p->stride_h | p->stride_s) & 7) != 0) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->S, (cuuint64_t)heads, (cuuint64_t)p->batch};
+    cuuint64_t strides[3] = {(cuuint64_t)p->stride_s * 2, (cuuint64_t)p->stride_h * 2, (cuuint64_t)p->stride_b * 2};
+    cuuint32_t box[4] = {64u, 32u, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(out), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 int launch_timeout_probe(const hilberta_plan_t *p, cudaStream_t stream) {
@@ -955,11 +1020,11 @@ int attn_bf16_prepare(hilberta_plan_t *p) {
         if (p->device < 0 || p->device >= 64) return HILBERTA_ERR_INVALID;
         if (!attr_done[p->device]) {
             HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128)));
-            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128, false, true)));
             HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64)));
-            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64, false, true)));
             HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<false, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128, true)));
-            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128, true)));
+            HB_CUDA(cudaFuncSetAttribute(attn_bf16_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128, true, true)));
             attr_done[p->device] = true;
         }
     }
@@ -1026,7 +1091,10 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
     prm.out_map = out_map;
     prm.lse = lse;
     prm.S = p->S;
+    // bit 0: 32-byte stores allowed; bit 1: rows leave through bulk tensor stores (physical order only)
     prm.out_align32 = (((uintptr_t)out & 31) == 0 && ((p->stride_b | p->stride_h | p->stride_s) & 15) == 0) ? 1 : 0;
+    CUtensorMap mo = mq;   // a valid map in any case; read only with bit 1 set
+    if (!in_map && !out_map && make_out_tensor_map(&mo, out, p, heads)) prm.out_align32 |= 2;
     if (in_map) {
         KernelParams<true> gprm;
         static_cast<Params &>(gprm) = prm;
@@ -1035,20 +1103,20 @@ int launch_attn_bf16(const hilberta_plan_t *p, const void *q, const void *k, con
         gprm.gk = k;
         gprm.gv = v;
         if (fp8)
-            attn_bf16_kernel<true, 128, true><<<n_cta, THREADS, smem_bytes(128, true), stream>>>(mq, mk, mv, gprm);
+            attn_bf16_kernel<true, 128, true><<<n_cta, THREADS, smem_bytes(128, true, true), stream>>>(mq, mk, mv, mo, gprm);
         else if (p->head_dim == 128)
-            attn_bf16_kernel<true, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, gprm);
+            attn_bf16_kernel<true, 128><<<n_cta, THREADS, smem_bytes(128, false, true), stream>>>(mq, mk, mv, mo, gprm);
         else
-            attn_bf16_kernel<true, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, gprm);
+            attn_bf16_kernel<true, 64><<<n_cta, THREADS, smem_bytes(64, false, true), stream>>>(mq, mk, mv, mo, gprm);
     } else {
         KernelParams<false> pprm;
         static_cast<Params &>(pprm) = prm;
         if (fp8)
-            attn_bf16_kernel<false, 128, true><<<n_cta, THREADS, smem_bytes(128, true), stream>>>(mq, mk, mv, pprm);
+            attn_bf16_kernel<false, 128, true><<<n_cta, THREADS, smem_bytes(128, true), stream>>>(mq, mk, mv, mo, pprm);
         else if (p->head_dim == 128)
-            attn_bf16_kernel<false, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, pprm);
+            attn_bf16_kernel<false, 128><<<n_cta, THREADS, smem_bytes(128), stream>>>(mq, mk, mv, mo, pprm);
         else
-            attn_bf16_kernel<false, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, pprm);
+            attn_bf16_kernel<false, 64><<<n_cta, THREADS, smem_bytes(64), stream>>>(mq, mk, mv, mo, pprm);
     }
     HB_LAUNCHED();
     return HILBERTA_OK;
