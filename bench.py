@@ -34,9 +34,10 @@ L2_BYTES = 126 * 2**20   # B200 L2
 COOL_DOWN_S = 1.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one forward launch: one ncu capture of the
-# single-CTA bf16 kernel at this workload, taken on the kernel revision that runs one-tile work items
-# for two heads at once (556.7 MB read + 94.9 MB written; the revision before it measured 647.5 MB).
-FORWARD_DRAM_TRAFFIC_BYTES = {"flux2048": 651.6e6}
+# single-CTA bf16 kernel at this workload, taken on the kernel revision with a four-slot K/V ring and
+# the output staging area (559.7 MB read + 99.7 MB written; the revisions before it measured 651.6 and
+# 647.5 MB).
+FORWARD_DRAM_TRAFFIC_BYTES = {"flux2048": 659.4e6}
 
 
 def load_peaks():

@@ -23,6 +23,10 @@
 // place by P_t (bf16, first 64 columns); O_t accumulators at [256 + 128 t, +128).
 // The running maximum is only advanced when it grows by more than 2^8, so the
 // O accumulator is rescaled rarely; exponentials stay below 2^8.
+// Shared memory: two Q tiles, a ring of K / V tiles, and (TMA instantiations) 32 KB in which the
+// softmax warps stage finished output rows, 4 KB per warp, for bulk tensor stores -- used where the
+// output keeps the physical order; scattered output (fused exit gather) and warps with rows beyond
+// the item store per lane.
 // FP8 instantiations take q, k, v as e4m3 bytes (128-byte rows, one slab per tile), round the
 // weights to e4m3 (four per TMEM column) and use kind::f8f6f4 MMAs; everything else is shared.
 #include <cuda.h>

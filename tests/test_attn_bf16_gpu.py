@@ -187,6 +187,36 @@ def test_forward_unpermute_equals_forward_then_unpermute():
             plan.destroy()
 
 
+@pytest.mark.parametrize("H,W,tile,o,hs,nt,D", [(24, 40, 256, 100, 4, 77, 128), (48, 32, 512, 256, 8, 130, 128),
+                                                 (5, 3, 16, 3, 2, 40, 128), (24, 40, 256, 100, 4, 77, 64),
+                                                 (64, 64, 1024, 512, 8, 512, 128)])
+def test_bulk_store_epilogue_equals_per_lane_epilogue(H, W, tile, o, hs, nt, D):
+    """Output in physical order leaves through shared memory and bulk tensor stores (warps whose 32
+    rows all belong to the work item) or through per-lane stores (ragged warps, scattered output):
+    both must write the same bits, also into a buffer that is only 16-byte aligned, and nothing
+    outside the tensor."""
+    S = nt + H * W
+    g = torch.Generator().manual_seed(99)
+    q, k, v = (torch.randn((2, 3, S, D), generator=g).bfloat16().cuda() for _ in range(3))
+    plan = hb.Plan(H, W, tile, o, hs, nt)
+    try:
+        plan.bind_like(q)
+        n = q.numel()
+        flat = torch.full((n + 64,), 7.0, dtype=torch.bfloat16, device="cuda")   # guard elements on both sides
+        out_phys = flat[8:8 + n].view(q.shape)                                     # base 16-byte aligned only
+        assert out_phys.data_ptr() % 32 == 16
+        out_a = torch.empty_like(q)
+        out_b = torch.full_like(q, float("nan"))
+        plan.forward(q, k, v, out_phys)
+        plan.unpermute(out_phys.contiguous(), out_a)
+        plan.forward_unpermute(q, k, v, out_b)
+        assert plan.status() == 0
+        assert torch.equal(out_a.view(torch.int16), out_b.view(torch.int16))
+        assert torch.all(flat[:8] == 7.0) and torch.all(flat[8 + n:] == 7.0)
+    finally:
+        plan.destroy()
+
+
 @pytest.mark.parametrize("H,W,tile,o,hs,nt", [(24, 40, 256, 100, 4, 77), (48, 32, 512, 256, 8, 130), (5, 3, 16, 3, 2, 40)])
 def test_general_shapes_elementwise(H, W, tile, o, hs, nt):
     """Non-square / non-power-of-two grids: same kernels, plan built on the padded curve."""
