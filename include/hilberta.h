@@ -280,8 +280,9 @@ int hilberta_backward_static(const void *dout, const void *q, const void *k, con
  * last attention layer of a step): q, k, v are in PHYSICAL order as for
  * hilberta_forward; `out` is written in ORIGINAL token order, i.e. physical row p
  * lands at row phys2orig[p].  Same layout, alignment, error and stream rules as
- * hilberta_forward.  Costs the same as hilberta_forward (each row is stored by one
- * thread either way) and saves the separate hilberta_unpermute pass. */
+ * hilberta_forward.  Costs about 2 % more than hilberta_forward (rows that go to
+ * scattered positions are stored per lane, rows that keep the physical order leave
+ * through bulk tensor stores) and saves the separate hilberta_unpermute pass. */
 int hilberta_forward_unpermute(const void *q, const void *k, const void *v, void *out,
                                const hilberta_plan_t *plan, void *stream);
 
